@@ -1,0 +1,220 @@
+/*
+ * adama.h -- C ABI of the B200 (sm_100a) AdamA optimizer library.
+ *
+ * AdamA (Adam Accumulation, arXiv 2305.19982) folds every micro-batch gradient
+ * straight into the Adam moments, so the gradient can be dropped as soon as it
+ * has been produced; at the end of the mini-batch a bias-corrected Adam update
+ * is applied.  One mini-batch, in the order of the paper's Algorithm 2:
+ *
+ *     adama_begin_minibatch(ctx, N)            t <- t+1; fixes N
+ *     for each micro-batch, for each layer (back to front):
+ *         adama_linear_wgrad_fold(...)         linear layers: G = X^T.dY is folded
+ *                                              from the tensor-core accumulator and
+ *                                              never written to memory
+ *         adama_fold(...)                      every other gradient tensor
+ *     for each parameter tensor:
+ *         adama_apply(...)                     update + beta-decay for the next step
+ *
+ * Conventions
+ *   - All tensor pointers are DEVICE pointers unless a parameter is named
+ *     *_host.  Memory is owned by the caller and only borrowed until the work
+ *     queued on `cuda_stream` has completed.  The library allocates its context,
+ *     a 256-byte device status block, one copy stream and a few events.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default
+ *     stream).  Calls are asynchronous and ordered by that stream.
+ *   - Gradients are passed RAW (as autograd produces them for one micro-batch);
+ *     the 1/N of Algorithm 2's "g <- (1/N) grad" is folded into the
+ *     coefficients a = (1-beta1)/N and b = (1-beta2)/N^2.  With the flag
+ *     ADAMA_GRADS_PRESCALED the caller has already divided by N and the
+ *     coefficients are a = 1-beta1, b = 1-beta2.
+ *   - State convention: Algorithm 2 decays m and v at the START of a
+ *     mini-batch.  This library performs that decay at the END of the previous
+ *     one, inside adama_apply, which stores beta1*m_t and beta2*v_t.  With
+ *     m_0 = v_0 = 0 the two orders give identical m_t, v_t and theta_t.  Between
+ *     adama_apply and the next fold the buffers therefore hold the decayed
+ *     moments; between the last fold and adama_apply they hold m_t and v_t.
+ *   - Hyper-parameters are doubles; every derived constant (1-beta, 1-beta^t,
+ *     lr/(1-beta1^t), ...) is formed in double on the host and rounded to fp32
+ *     once.
+ *   - One context per model replica.  A context is not thread-safe.
+ *   - Every function returns an adama_status; nothing aborts, traps or prints.
+ *     adama_last_error gives a message for the last failing call on a context.
+ */
+#ifndef ADAMA_H_
+#define ADAMA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define ADAMA_API __attribute__((visibility("default")))
+#else
+#define ADAMA_API
+#endif
+
+typedef struct adama_ctx adama_ctx; /* opaque; created by adama_init, freed by adama_destroy */
+
+typedef enum adama_status {
+    ADAMA_OK = 0,
+    ADAMA_ERR_INVALID_ARG = 1, /* null pointer, negative size, N < 1, bad hyper-parameter      */
+    ADAMA_ERR_BAD_STATE = 2,   /* call order: fold/apply before the first begin_minibatch      */
+    ADAMA_ERR_MISALIGNED = 3,  /* pointer or pitch violates the alignment stated for the call  */
+    ADAMA_ERR_UNSUPPORTED = 4, /* device is not sm_100, or a size exceeds a documented limit   */
+    ADAMA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed; see adama_last_error      */
+    ADAMA_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by sync_status) */
+} adama_status;
+
+typedef enum adama_dtype { ADAMA_F32 = 0, ADAMA_BF16 = 1 } adama_dtype;
+
+/* flags for adama_config.flags */
+#define ADAMA_GRADS_PRESCALED 1u /* gradients already carry the 1/N of Algorithm 2 */
+
+typedef struct adama_config {
+    double beta1;   /* in [0,1)                                    */
+    double beta2;   /* in [0,1)                                    */
+    double eps;     /* >= 0; added outside the square root         */
+    int device;     /* CUDA device ordinal the context is bound to */
+    unsigned flags; /* ADAMA_* flags                               */
+} adama_config;
+
+/* Algorithm 2, "Initialize": t <- 0.  (theta_0, m_0 = 0 and v_0 = 0 are the
+ * caller's buffers: the caller zero-fills m and v once.)  Creates the context
+ * on cfg->device, which must be a compute-capability-10.x GPU; the device's
+ * primary context is initialised if needed.  Allocates a 256-byte device
+ * status block, a copy stream and a few events.
+ * Errors: INVALID_ARG (null, betas outside [0,1), eps < 0), UNSUPPORTED (not
+ * sm_100), CUDA. */
+ADAMA_API adama_status adama_init(adama_ctx **out, const adama_config *cfg);
+
+/* Frees everything adama_init allocated.  The caller must have synchronised
+ * the streams it used.  NULL is accepted. */
+ADAMA_API adama_status adama_destroy(adama_ctx *ctx);
+
+/* Algorithm 2, first line of the loop body: t <- t+1, and N (micro-batches in
+ * this mini-batch, >= 1) is fixed, which fixes a = (1-beta1)/N and
+ * b = (1-beta2)/N^2 for every fold until the next call.  Host-only, no GPU
+ * work: the decay "m <- beta1 m, v <- beta2 v" of the same line was already
+ * applied by the previous adama_apply (see "State convention").
+ * Errors: INVALID_ARG (n_micro < 1). */
+ADAMA_API adama_status adama_begin_minibatch(adama_ctx *ctx, int n_micro);
+
+/* Algorithm 2, inner loop body for one (micro-batch, layer):
+ *     m <- m + (1-beta1) g,   v <- v + (1-beta2) g^2,   g = grad / N
+ * computed as m += a*grad, v += b*grad^2 in fp32 (one FMA each).
+ *   grad : n elements, dtype gdt (fp32 or bf16), contiguous, device, read-only
+ *   m, v : n fp32 elements each, contiguous, device, updated in place
+ * Any n >= 0 and any element-aligned pointers are accepted: the kernel uses
+ * 128-bit accesses when grad, m and v allow it and a scalar path otherwise.
+ * m and v must not overlap each other or grad.
+ * Errors: INVALID_ARG, BAD_STATE (no begin_minibatch yet), MISALIGNED (pointer
+ * not aligned to its element size), CUDA (launch failure). */
+ADAMA_API adama_status adama_fold(adama_ctx *ctx, const void *grad, adama_dtype gdt, float *m,
+                                  float *v, size_t n, void *cuda_stream);
+
+/* The same accumulation for a linear layer y = x.W, W of shape [d_in, d_out],
+ * whose raw weight gradient is G = X^T.dY ("once the gradients of a layer are
+ * produced" in Section 3.1; Algorithm 2's "assign / release memory for g"
+ * disappears because G only ever exists as a tensor-memory accumulator tile):
+ *     G[p,q] = sum_{tau < tokens} X[tau,p] * dY[tau,q]   (bf16 x bf16 -> fp32)
+ *     m[p,q] += a*G[p,q],   v[p,q] += b*G[p,q]^2
+ *   X    : [tokens, d_in]  bf16 row-major, row pitch ldx  elements, device, read-only
+ *   dY   : [tokens, d_out] bf16 row-major, row pitch ldy  elements, device, read-only
+ *   m, v : [d_in, d_out]   fp32 row-major, row pitch ldmv elements, device, in place
+ * Requirements (checked, MISALIGNED / INVALID_ARG otherwise): X, dY, m, v
+ * 16-byte aligned; ldx, ldy multiples of 8; ldmv a multiple of 4; ldx >= d_in,
+ * ldy >= d_out, ldmv >= d_out; d_in, d_out >= 1; tokens >= 0 (0 is a no-op).
+ * Any d_in, d_out, tokens within those rules are handled (ragged tiles are
+ * zero-filled on load and clipped on store).  The whole token sum of one call
+ * is finished before it is squared: there is no split over tokens.
+ * m and v are updated by tile-wise reduce-add through the L2; each element is
+ * touched exactly once per call, so results do not depend on scheduling.
+ * A caller that stores W as [d_out, d_in] passes (dY, X) in place of (X, dY).
+ * Device-side waits are bounded; if one expires the kernel stops early, leaves
+ * a code in the status block and adama_sync_status returns ADAMA_ERR_TIMEOUT.
+ * Errors: INVALID_ARG, BAD_STATE, MISALIGNED, UNSUPPORTED, CUDA. */
+ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *dY,
+                                               int tokens, int d_in, int d_out, int64_t ldx,
+                                               int64_t ldy, float *m, float *v, int64_t ldmv,
+                                               void *cuda_stream);
+
+/* Algorithm 2, "Update", fused with the first line of the NEXT loop body:
+ *     m_hat = m/(1-beta1^t), v_hat = v/(1-beta2^t),
+ *     w <- w - lr * m_hat / (sqrt(v_hat) + eps)
+ *     m <- beta1*m, v <- beta2*v            (decay for mini-batch t+1)
+ *   w, m, v : n fp32 elements each, contiguous, device, updated in place.
+ * `lr` is the step size alpha of this mini-batch (schedules stay with the
+ * caller).  Call once per parameter tensor per mini-batch, after its last fold.
+ * Errors: INVALID_ARG, BAD_STATE (t == 0), MISALIGNED, CUDA. */
+ADAMA_API adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
+                                   double lr, void *cuda_stream);
+
+/* ---- host-buffer variants (same arithmetic, copies included) --------------------------- */
+
+/* adama_fold with the gradient in HOST memory (pinned memory for full copy
+ * speed).  The gradient is streamed through `staging` (device, caller-owned,
+ * staging_bytes >= 2 MiB, 256-byte aligned) in two alternating halves on the
+ * context's copy stream while the fold of the previous half runs on
+ * `cuda_stream`.  On return all work is queued; grad_host and staging are
+ * borrowed until `cuda_stream` has completed. */
+ADAMA_API adama_status adama_fold_host(adama_ctx *ctx, const void *grad_host, adama_dtype gdt,
+                                       float *m, float *v, size_t n, void *staging,
+                                       size_t staging_bytes, void *cuda_stream);
+
+/* adama_linear_wgrad_fold with X and dY in HOST memory, dense (ldx = d_in,
+ * ldy = d_out, both multiples of 8).  Both are copied into `staging` (device,
+ * caller-owned, at least 2*tokens*(d_in+d_out) + 256 bytes, 256-byte aligned)
+ * on `cuda_stream`, then the fused kernel runs. */
+ADAMA_API adama_status adama_linear_wgrad_fold_host(adama_ctx *ctx, const void *X_host,
+                                                    const void *dY_host, int tokens, int d_in,
+                                                    int d_out, float *m, float *v, int64_t ldmv,
+                                                    void *staging, size_t staging_bytes,
+                                                    void *cuda_stream);
+
+/* adama_apply followed by a device-to-host copy of the updated weights into
+ * w_host (n fp32, pinned memory for full speed), queued on `cuda_stream`. */
+ADAMA_API adama_status adama_apply_to_host(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
+                                           double lr, float *w_host, void *cuda_stream);
+
+/* ---- state, checkpointing, diagnostics ------------------------------------------------- */
+
+/* Step counter t of Algorithm 2 (0 after init). */
+ADAMA_API int64_t adama_get_step(const adama_ctx *ctx);
+/* Restore t from a checkpoint (t >= 0).  The saved m, v must follow the state
+ * convention above (decayed if saved after adama_apply). */
+ADAMA_API adama_status adama_set_step(adama_ctx *ctx, int64_t t);
+/* Micro-batch count fixed by the last begin_minibatch (0 before the first). */
+ADAMA_API int adama_get_n_micro(const adama_ctx *ctx);
+
+/* Waits for `cuda_stream`, then reads and clears the device status block.
+ * Returns ADAMA_OK, ADAMA_ERR_TIMEOUT (a bounded wait inside the fused kernel
+ * expired; m and v of that call are incomplete) or ADAMA_ERR_CUDA. */
+ADAMA_API adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream);
+
+/* Message for the most recent non-OK status returned on this context ("" if
+ * none).  The pointer stays valid until the next call on the context. */
+ADAMA_API const char *adama_last_error(const adama_ctx *ctx);
+
+/* Number of kernels this context has launched since adama_init. */
+ADAMA_API int64_t adama_launch_count(const adama_ctx *ctx);
+
+/* Host-only, no GPU needed: the fp32 constants the kernels receive for a given
+ * configuration, N, step t (>= 1) and lr, each derived in double from
+ * Algorithm 2 and rounded once:
+ *   out[0] = a = (1-beta1)/N          out[1] = b = (1-beta2)/N^2
+ *   out[2] = lr/(1-beta1^t)           out[3] = 1/(1-beta2^t)        out[4] = eps
+ *   out[5], out[6] = beta1 split as hi + lo   out[7], out[8] = beta2 split as hi + lo
+ * Errors: INVALID_ARG. */
+ADAMA_API adama_status adama_host_constants(const adama_config *cfg, int n_micro, int64_t t,
+                                            double lr, float out[9]);
+
+/* Library version, "major.minor.patch". */
+ADAMA_API const char *adama_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAMA_H_ */
