@@ -1,0 +1,402 @@
+// C ABI of libadama: context, argument checks, host-side constants, launches.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "adama_internal.h"
+
+struct adama_ctx {
+    adama_config cfg;
+    int64_t t;    // step counter of Algorithm 2
+    int n_micro;  // N of the current mini-batch (0 before the first)
+    adama::FoldConstants fold_c;
+    int sm_count;
+    unsigned *status_dev;      // 256-byte device status block
+    cudaStream_t copy_stream;  // host-buffer variants: H2D copies overlap the folds
+    cudaEvent_t ev_copied[2], ev_folded[2], ev_entry;
+    int64_t launches;
+    char err[256];
+};
+
+namespace adama {
+
+FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsigned flags) {
+    double N = (flags & ADAMA_GRADS_PRESCALED) ? 1.0 : (double)n_micro;
+    FoldConstants c;
+    c.a = (float)((1.0 - beta1) / N);
+    c.b = (float)((1.0 - beta2) / (N * N));
+    return c;
+}
+
+static void split_hi_lo(double x, float *hi, float *lo) {
+    *hi = (float)x;
+    *lo = (float)(x - (double)*hi);
+}
+
+ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr) {
+    ApplyConstants c;
+    double bc1 = 1.0 - pow(beta1, (double)t);
+    double bc2 = 1.0 - pow(beta2, (double)t);
+    c.step = (float)(lr / bc1);
+    c.inv_bc2 = (float)(1.0 / bc2);
+    c.eps = (float)eps;
+    split_hi_lo(beta1, &c.beta1_hi, &c.beta1_lo);
+    split_hi_lo(beta2, &c.beta2_hi, &c.beta2_lo);
+    return c;
+}
+
+}  // namespace adama
+
+namespace {
+
+adama_status fail(adama_ctx *ctx, adama_status st, const char *msg) {
+    if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
+    return st;
+}
+
+adama_status cuda_fail(adama_ctx *ctx, const char *what, cudaError_t e) {
+    if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s: %s", what, cudaGetErrorString(e));
+    return ADAMA_ERR_CUDA;
+}
+
+bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Makes ctx's device current for the duration of a call and restores the caller's.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+size_t dtype_size(adama_dtype d) { return d == ADAMA_F32 ? 4 : 2; }
+
+bool config_ok(const adama_config *cfg) {
+    return cfg && cfg->beta1 >= 0.0 && cfg->beta1 < 1.0 && cfg->beta2 >= 0.0 && cfg->beta2 < 1.0 &&
+           cfg->eps >= 0.0 && isfinite(cfg->eps) && cfg->device >= 0 &&
+           (cfg->flags & ~ADAMA_GRADS_PRESCALED) == 0;
+}
+
+adama_status check_fold_args(adama_ctx *ctx, const void *grad, adama_dtype gdt, float *m, float *v,
+                             size_t n) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (gdt != ADAMA_F32 && gdt != ADAMA_BF16)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "fold: unknown gradient dtype");
+    if (n > 0 && (!grad || !m || !v)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "fold: null pointer");
+    if (ctx->n_micro < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "fold: adama_begin_minibatch has not been called");
+    if (!aligned_to(grad, dtype_size(gdt)) || !aligned_to(m, 4) || !aligned_to(v, 4))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "fold: pointer not aligned to its element size");
+    return ADAMA_OK;
+}
+
+adama_status check_wgrad_args(adama_ctx *ctx, const void *X, const void *dY, int tokens, int d_in,
+                              int d_out, int64_t ldx, int64_t ldy, float *m, float *v,
+                              int64_t ldmv) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (tokens < 0 || d_in < 1 || d_out < 1)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold: bad shape");
+    if (!m || !v || (tokens > 0 && (!X || !dY)))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold: null pointer");
+    if (ldx < d_in || ldy < d_out || ldmv < d_out)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold: row pitch smaller than the row");
+    if (ctx->n_micro < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "wgrad_fold: adama_begin_minibatch has not been called");
+    if (!aligned_to(X, 16) || !aligned_to(dY, 16) || !aligned_to(m, 16) || !aligned_to(v, 16))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "wgrad_fold: X, dY, m, v must be 16-byte aligned");
+    if (ldx % 8 || ldy % 8 || ldmv % 4)
+        return fail(ctx, ADAMA_ERR_MISALIGNED,
+                    "wgrad_fold: ldx, ldy must be multiples of 8 and ldmv of 4");
+    // tensor-map strides are limited to 2^40 bytes
+    if (ldx * 2 >= (1ll << 40) || ldy * 2 >= (1ll << 40) || ldmv * 4 >= (1ll << 40))
+        return fail(ctx, ADAMA_ERR_UNSUPPORTED, "wgrad_fold: row pitch too large for a tensor map");
+    return ADAMA_OK;
+}
+
+adama_status check_apply_args(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (n > 0 && (!w || !m || !v)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply: null pointer");
+    if (!isfinite(lr)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply: lr is not finite");
+    if (ctx->t < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "apply: no mini-batch has been started (t == 0)");
+    if (!aligned_to(w, 4) || !aligned_to(m, 4) || !aligned_to(v, 4))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "apply: pointer not aligned to 4 bytes");
+    return ADAMA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *adama_version(void) { return "0.1.0"; }
+
+adama_status adama_init(adama_ctx **out, const adama_config *cfg) {
+    if (!out) return ADAMA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!config_ok(cfg)) return ADAMA_ERR_INVALID_ARG;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || cfg->device >= count) return ADAMA_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return ADAMA_ERR_CUDA;
+    if (prop.major != 10) return ADAMA_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+
+    adama_ctx *ctx = new (std::nothrow) adama_ctx();
+    if (!ctx) return ADAMA_ERR_CUDA;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->cfg = *cfg;
+    ctx->sm_count = prop.multiProcessorCount;
+
+    DeviceGuard guard(cfg->device);
+    const char *msg = "";
+    cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->status_dev), 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->status_dev, 0, 256);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming);
+        if (e == cudaSuccess)
+            e = cudaEventCreateWithFlags(&ctx->ev_folded[i], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = adama::wgrad_fold_setup(&msg);
+    if (e != cudaSuccess) {
+        adama_destroy(ctx);
+        return ADAMA_ERR_CUDA;
+    }
+    *out = ctx;
+    return ADAMA_OK;
+}
+
+adama_status adama_destroy(adama_ctx *ctx) {
+    if (!ctx) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (ctx->status_dev) cudaFree(ctx->status_dev);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
+        if (ctx->ev_folded[i]) cudaEventDestroy(ctx->ev_folded[i]);
+    }
+    if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+    delete ctx;
+    return ADAMA_OK;
+}
+
+adama_status adama_begin_minibatch(adama_ctx *ctx, int n_micro) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (n_micro < 1) return fail(ctx, ADAMA_ERR_INVALID_ARG, "begin_minibatch: n_micro must be >= 1");
+    ctx->t += 1;
+    ctx->n_micro = n_micro;
+    ctx->fold_c = adama::make_fold_constants(ctx->cfg.beta1, ctx->cfg.beta2, n_micro, ctx->cfg.flags);
+    return ADAMA_OK;
+}
+
+adama_status adama_fold(adama_ctx *ctx, const void *grad, adama_dtype gdt, float *m, float *v,
+                        size_t n, void *cuda_stream) {
+    adama_status st = check_fold_args(ctx, grad, gdt, m, v, n);
+    if (st != ADAMA_OK) return st;
+    if (n == 0) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaError_t e = adama::launch_fold(grad, gdt, m, v, n, ctx->fold_c, ctx->sm_count,
+                                       static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "fold launch", e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
+adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *dY, int tokens,
+                                     int d_in, int d_out, int64_t ldx, int64_t ldy, float *m,
+                                     float *v, int64_t ldmv, void *cuda_stream) {
+    adama_status st = check_wgrad_args(ctx, X, dY, tokens, d_in, d_out, ldx, ldy, m, v, ldmv);
+    if (st != ADAMA_OK) return st;
+    if (tokens == 0) return ADAMA_OK;  // empty sum: G = 0, nothing to add
+    DeviceGuard guard(ctx->cfg.device);
+    adama::WgradArgs a;
+    a.X = X;
+    a.dY = dY;
+    a.tokens = tokens;
+    a.d_in = d_in;
+    a.d_out = d_out;
+    a.ldx = ldx;
+    a.ldy = ldy;
+    a.ldmv = ldmv;
+    a.m = m;
+    a.v = v;
+    a.c = ctx->fold_c;
+    a.status = ctx->status_dev;
+    a.sm_count = ctx->sm_count;
+    a.stream = static_cast<cudaStream_t>(cuda_stream);
+    const char *msg = "wgrad_fold";
+    cudaError_t e = adama::launch_wgrad_fold(a, &msg);
+    if (e != cudaSuccess) return cuda_fail(ctx, msg, e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
+adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
+                         void *cuda_stream) {
+    adama_status st = check_apply_args(ctx, w, m, v, n, lr);
+    if (st != ADAMA_OK) return st;
+    if (n == 0) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    adama::ApplyConstants c =
+        adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr);
+    cudaError_t e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "apply launch", e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
+// ---- host-buffer variants -------------------------------------------------------------------
+
+adama_status adama_fold_host(adama_ctx *ctx, const void *grad_host, adama_dtype gdt, float *m,
+                             float *v, size_t n, void *staging, size_t staging_bytes,
+                             void *cuda_stream) {
+    adama_status st = check_fold_args(ctx, grad_host, gdt, m, v, n);
+    if (st != ADAMA_OK) return st;
+    if (n == 0) return ADAMA_OK;
+    if (!staging || staging_bytes < (2u << 20))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "fold_host: staging buffer smaller than 2 MiB");
+    if (!aligned_to(staging, 256))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "fold_host: staging must be 256-byte aligned");
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t esz = dtype_size(gdt);
+    // two halves, each a multiple of 256 bytes, so every chunk keeps m, v and grad 16-byte aligned
+    const size_t half_bytes = (staging_bytes / 2) & ~(size_t)255;
+    const size_t chunk = half_bytes / esz;
+    char *half[2] = {static_cast<char *>(staging), static_cast<char *>(staging) + half_bytes};
+    const char *src = static_cast<const char *>(grad_host);
+
+    // the staging buffer may still be in use by earlier work on `stream`
+    cudaError_t e = cudaEventRecord(ctx->ev_entry, stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_entry, 0);
+    size_t done = 0;
+    for (int it = 0; done < n && e == cudaSuccess; ++it) {
+        const int h = it & 1;
+        const size_t cnt = (n - done < chunk) ? (n - done) : chunk;
+        if (it >= 2) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_folded[h], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(half[h], src + done * esz, cnt * esz, cudaMemcpyHostToDevice,
+                                ctx->copy_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_copied[h], ctx->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_copied[h], 0);
+        if (e == cudaSuccess) {
+            e = adama::launch_fold(half[h], gdt, m + done, v + done, cnt, ctx->fold_c,
+                                   ctx->sm_count, stream);
+            ctx->launches += 1;
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_folded[h], stream);
+        done += cnt;
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, "fold_host", e);
+    return ADAMA_OK;
+}
+
+adama_status adama_linear_wgrad_fold_host(adama_ctx *ctx, const void *X_host, const void *dY_host,
+                                          int tokens, int d_in, int d_out, float *m, float *v,
+                                          int64_t ldmv, void *staging, size_t staging_bytes,
+                                          void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (tokens < 0 || d_in < 1 || d_out < 1)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold_host: bad shape");
+    if (d_in % 8 || d_out % 8)
+        return fail(ctx, ADAMA_ERR_MISALIGNED,
+                    "wgrad_fold_host: dense rows need d_in, d_out multiples of 8");
+    const size_t x_bytes = (size_t)tokens * d_in * 2, y_bytes = (size_t)tokens * d_out * 2;
+    const size_t y_off = (x_bytes + 255) & ~(size_t)255;
+    if (!staging || staging_bytes < y_off + y_bytes)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold_host: staging buffer too small");
+    if (!aligned_to(staging, 256))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "wgrad_fold_host: staging must be 256-byte aligned");
+    char *Xd = static_cast<char *>(staging), *Yd = Xd + y_off;
+    adama_status st = check_wgrad_args(ctx, Xd, Yd, tokens, d_in, d_out, d_in, d_out, m, v, ldmv);
+    if (st != ADAMA_OK) return st;
+    if (tokens == 0) return ADAMA_OK;
+    if (!X_host || !dY_host) return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold_host: null pointer");
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemcpyAsync(Xd, X_host, x_bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(Yd, dY_host, y_bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, "wgrad_fold_host copy", e);
+    return adama_linear_wgrad_fold(ctx, Xd, Yd, tokens, d_in, d_out, d_in, d_out, m, v, ldmv,
+                                   cuda_stream);
+}
+
+adama_status adama_apply_to_host(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
+                                 float *w_host, void *cuda_stream) {
+    if (ctx && n > 0 && !w_host)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply_to_host: null host pointer");
+    adama_status st = adama_apply(ctx, w, m, v, n, lr, cuda_stream);
+    if (st != ADAMA_OK || n == 0) return st;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaError_t e = cudaMemcpyAsync(w_host, w, n * sizeof(float), cudaMemcpyDeviceToHost,
+                                    static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "apply_to_host copy", e);
+    return ADAMA_OK;
+}
+
+// ---- state and diagnostics ------------------------------------------------------------------
+
+int64_t adama_get_step(const adama_ctx *ctx) { return ctx ? ctx->t : -1; }
+
+adama_status adama_set_step(adama_ctx *ctx, int64_t t) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (t < 0) return fail(ctx, ADAMA_ERR_INVALID_ARG, "set_step: t must be >= 0");
+    ctx->t = t;
+    return ADAMA_OK;
+}
+
+int adama_get_n_micro(const adama_ctx *ctx) { return ctx ? ctx->n_micro : -1; }
+
+adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned host[4] = {0, 0, 0, 0};
+    cudaError_t e =
+        cudaMemcpyAsync(host, ctx->status_dev, sizeof(host), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, "sync_status", e);
+    if (host[0] != adama::kDevOk) {
+        e = cudaMemsetAsync(ctx->status_dev, 0, 256, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+        snprintf(ctx->err, sizeof(ctx->err),
+                 "device-side wait expired in the fused weight-gradient kernel "
+                 "(code %u, wait %u, tile %u)",
+                 host[0], host[1], host[2]);
+        return ADAMA_ERR_TIMEOUT;
+    }
+    return ADAMA_OK;
+}
+
+const char *adama_last_error(const adama_ctx *ctx) { return ctx ? ctx->err : ""; }
+
+int64_t adama_launch_count(const adama_ctx *ctx) { return ctx ? ctx->launches : -1; }
+
+adama_status adama_host_constants(const adama_config *cfg, int n_micro, int64_t t, double lr,
+                                  float out[9]) {
+    if (!config_ok(cfg) || !out || n_micro < 1 || t < 1) return ADAMA_ERR_INVALID_ARG;
+    adama::FoldConstants f = adama::make_fold_constants(cfg->beta1, cfg->beta2, n_micro, cfg->flags);
+    adama::ApplyConstants c = adama::make_apply_constants(cfg->beta1, cfg->beta2, cfg->eps, t, lr);
+    out[0] = f.a;
+    out[1] = f.b;
+    out[2] = c.step;
+    out[3] = c.inv_bc2;
+    out[4] = c.eps;
+    out[5] = c.beta1_hi;
+    out[6] = c.beta1_lo;
+    out[7] = c.beta2_hi;
+    out[8] = c.beta2_lo;
+    return ADAMA_OK;
+}
+
+}  // extern "C"

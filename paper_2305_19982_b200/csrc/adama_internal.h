@@ -1,0 +1,61 @@
+// Internal declarations shared by the translation units of libadama (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "adama.h"
+
+namespace adama {
+
+// Constants of one mini-batch / one update, derived in double on the host and
+// rounded to fp32 once (forming 1-beta2 in fp32 would already cost 1e-5
+// relative accuracy on v).
+struct FoldConstants {
+    float a;  // (1-beta1)/N     (or 1-beta1 with ADAMA_GRADS_PRESCALED)
+    float b;  // (1-beta2)/N^2   (or 1-beta2)
+};
+
+struct ApplyConstants {
+    float step;      // lr / (1 - beta1^t)
+    float inv_bc2;   // 1 / (1 - beta2^t)
+    float eps;       // eps
+    float beta1_hi;  // beta1 = beta1_hi + beta1_lo to ~1e-15: the decay m*beta1 is
+    float beta1_lo;  // formed as fma(m, lo, m*hi), free of a per-step bias that
+    float beta2_hi;  // would otherwise build up over ~1/(1-beta) steps
+    float beta2_lo;
+};
+
+FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsigned flags);
+ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr);
+
+// Status block in device memory (256 bytes): word 0 = first error code recorded
+// by a kernel (0 = none), word 1 = which wait, word 2 = tile; rest reserved.
+enum DeviceErr : unsigned { kDevOk = 0, kDevTimeout = 1 };
+
+// streaming kernels (fold_apply.cu)
+cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, size_t n,
+                        FoldConstants c, int sm_count, cudaStream_t stream);
+cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants c, int sm_count,
+                         cudaStream_t stream);
+
+// fused weight-gradient + fold (wgrad_fold.cu)
+struct WgradArgs {
+    const void *X;
+    const void *dY;
+    int tokens, d_in, d_out;
+    int64_t ldx, ldy, ldmv;
+    float *m;
+    float *v;
+    FoldConstants c;
+    unsigned *status;  // device status block
+    int sm_count;
+    cudaStream_t stream;
+};
+// Returns cudaSuccess or the failing CUDA error; *msg (static string) says which step failed.
+cudaError_t launch_wgrad_fold(const WgradArgs &args, const char **msg);
+// One-time, per process: resolves the driver's tensor-map encoder.
+cudaError_t wgrad_fold_setup(const char **msg);
+
+}  // namespace adama

@@ -1,0 +1,246 @@
+// Streaming kernels of AdamA: the moment fold (Algorithm 2, inner loop body) and
+// the update fused with the next mini-batch's decay (Algorithm 2, "Update" and the
+// first line of the loop body).  Both are pure HBM streams: one pass, every byte
+// touched once, 128-bit coalesced accesses, several independent loads in flight
+// per thread, grid sized as a multiple of the SM count with a grid-stride loop.
+#include <cuda_bf16.h>
+
+#include "adama_internal.h"
+
+namespace adama {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kCtasPerSm = 4;       // fold: 4 x 256 threads, <= 64 registers each
+constexpr int kApplyCtasPerSm = 3;  // apply holds 48 data registers per thread: <= 85 each
+
+// ---- 128-bit global accesses ------------------------------------------------------------
+// m, v and w are read once and written once per pass, the gradient is read once:
+// loads do not allocate in L1.
+__device__ __forceinline__ float4 ld_stream(const float4 *p) {
+    float4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "l"(p));
+    return r;
+}
+__device__ __forceinline__ uint2 ld_stream_ro(const uint2 *p) {
+    uint2 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ float4 ld_stream_ro(const float4 *p) {
+    float4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_stream(float4 *p, float4 x) {
+    asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z),
+                 "f"(x.w)
+                 : "memory");
+}
+
+// four gradient values widened exactly to fp32
+struct Grad4 {
+    float x, y, z, w;
+};
+__device__ __forceinline__ Grad4 load_grad4(const float *g, size_t i4) {
+    float4 t = ld_stream_ro(reinterpret_cast<const float4 *>(g) + i4);
+    return {t.x, t.y, t.z, t.w};
+}
+__device__ __forceinline__ Grad4 load_grad4(const __nv_bfloat16 *g, size_t i4) {
+    uint2 t = ld_stream_ro(reinterpret_cast<const uint2 *>(g) + i4);
+    // bf16 -> fp32 is a 16-bit left shift
+    return {__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
+            __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u)};
+}
+__device__ __forceinline__ float widen(float g) { return g; }
+__device__ __forceinline__ float widen(__nv_bfloat16 g) { return __bfloat162float(g); }
+
+// m += a*g ; v += b*g^2      (Algorithm 2: m += (1-beta1) g/N, v += (1-beta2) (g/N)^2)
+__device__ __forceinline__ void fold1(float g, float &m, float &v, float a, float b) {
+    m = fmaf(a, g, m);
+    v = fmaf(b * g, g, v);
+}
+
+template <typename G, int UNROLL>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+fold_vec_kernel(const G *__restrict__ grad, float *__restrict__ m, float *__restrict__ v,
+                size_t n4, size_t n, float a, float b) {
+    float4 *m4 = reinterpret_cast<float4 *>(m);
+    float4 *v4 = reinterpret_cast<float4 *>(v);
+    const size_t span = (size_t)kThreads * UNROLL;
+    for (size_t base = (size_t)blockIdx.x * span; base < n4; base += (size_t)gridDim.x * span) {
+        Grad4 g[UNROLL];
+        float4 mm[UNROLL], vv[UNROLL];
+        // all loads of the iteration are issued before the first use
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            size_t i = base + (size_t)u * kThreads + threadIdx.x;
+            if (i < n4) {
+                g[u] = load_grad4(grad, i);
+                mm[u] = ld_stream(m4 + i);
+                vv[u] = ld_stream(v4 + i);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            size_t i = base + (size_t)u * kThreads + threadIdx.x;
+            if (i < n4) {
+                fold1(g[u].x, mm[u].x, vv[u].x, a, b);
+                fold1(g[u].y, mm[u].y, vv[u].y, a, b);
+                fold1(g[u].z, mm[u].z, vv[u].z, a, b);
+                fold1(g[u].w, mm[u].w, vv[u].w, a, b);
+                st_stream(m4 + i, mm[u]);
+                st_stream(v4 + i, vv[u]);
+            }
+        }
+    }
+    // ragged tail (n not a multiple of 4): at most 3 elements
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - n4 * 4)) {
+        size_t i = n4 * 4 + threadIdx.x;
+        float mi = m[i], vi = v[i];
+        fold1(widen(grad[i]), mi, vi, a, b);
+        m[i] = mi;
+        v[i] = vi;
+    }
+}
+
+// Fallback for pointers that are not 16-byte aligned (8-byte for bf16 gradients).
+template <typename G>
+__global__ void __launch_bounds__(kThreads)
+fold_scalar_kernel(const G *__restrict__ grad, float *__restrict__ m, float *__restrict__ v,
+                   size_t n, float a, float b) {
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n;
+         i += (size_t)gridDim.x * kThreads) {
+        float mi = m[i], vi = v[i];
+        fold1(widen(grad[i]), mi, vi, a, b);
+        m[i] = mi;
+        v[i] = vi;
+    }
+}
+
+// w -= step * m / (sqrt(v*inv_bc2) + eps);  m *= beta1;  v *= beta2
+__device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
+    float denom = sqrtf(v * c.inv_bc2) + c.eps;  // IEEE sqrt
+    w = fmaf(-c.step, m / denom, w);             // IEEE division
+    m = fmaf(m, c.beta1_lo, m * c.beta1_hi);
+    v = fmaf(v, c.beta2_lo, v * c.beta2_hi);
+}
+
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads, kApplyCtasPerSm)
+apply_vec_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict__ v, size_t n4,
+                 size_t n, ApplyConstants c) {
+    float4 *w4 = reinterpret_cast<float4 *>(w);
+    float4 *m4 = reinterpret_cast<float4 *>(m);
+    float4 *v4 = reinterpret_cast<float4 *>(v);
+    const size_t span = (size_t)kThreads * UNROLL;
+    for (size_t base = (size_t)blockIdx.x * span; base < n4; base += (size_t)gridDim.x * span) {
+        float4 ww[UNROLL], mm[UNROLL], vv[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            size_t i = base + (size_t)u * kThreads + threadIdx.x;
+            if (i < n4) {
+                ww[u] = ld_stream(w4 + i);
+                mm[u] = ld_stream(m4 + i);
+                vv[u] = ld_stream(v4 + i);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            size_t i = base + (size_t)u * kThreads + threadIdx.x;
+            if (i < n4) {
+                apply1(ww[u].x, mm[u].x, vv[u].x, c);
+                apply1(ww[u].y, mm[u].y, vv[u].y, c);
+                apply1(ww[u].z, mm[u].z, vv[u].z, c);
+                apply1(ww[u].w, mm[u].w, vv[u].w, c);
+                st_stream(w4 + i, ww[u]);
+                st_stream(m4 + i, mm[u]);
+                st_stream(v4 + i, vv[u]);
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - n4 * 4)) {
+        size_t i = n4 * 4 + threadIdx.x;
+        float wi = w[i], mi = m[i], vi = v[i];
+        apply1(wi, mi, vi, c);
+        w[i] = wi;
+        m[i] = mi;
+        v[i] = vi;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+apply_scalar_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict__ v, size_t n,
+                    ApplyConstants c) {
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n;
+         i += (size_t)gridDim.x * kThreads) {
+        float wi = w[i], mi = m[i], vi = v[i];
+        apply1(wi, mi, vi, c);
+        w[i] = wi;
+        m[i] = mi;
+        v[i] = vi;
+    }
+}
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Grid: enough CTAs to cover the data once, capped at a whole number of CTAs per SM.
+inline unsigned grid_for(size_t work_items, size_t items_per_cta, int sm_count,
+                         int ctas_per_sm = kCtasPerSm) {
+    size_t need = (work_items + items_per_cta - 1) / items_per_cta;
+    size_t cap = (size_t)sm_count * ctas_per_sm;
+    if (need < 1) need = 1;
+    return (unsigned)(need < cap ? need : cap);
+}
+
+}  // namespace
+
+cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, size_t n,
+                        FoldConstants c, int sm_count, cudaStream_t stream) {
+    if (n == 0) return cudaSuccess;
+    constexpr int U = 4;
+    const size_t n4 = n / 4;
+    const bool vec = aligned(m, 16) && aligned(v, 16) && aligned(grad, gdt == ADAMA_F32 ? 16 : 8);
+    if (gdt == ADAMA_F32) {
+        const float *g = static_cast<const float *>(grad);
+        if (vec) {
+            unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count);
+            fold_vec_kernel<float, U><<<grid, kThreads, 0, stream>>>(g, m, v, n4, n, c.a, c.b);
+        } else {
+            unsigned grid = grid_for(n, kThreads, sm_count);
+            fold_scalar_kernel<float><<<grid, kThreads, 0, stream>>>(g, m, v, n, c.a, c.b);
+        }
+    } else {
+        const __nv_bfloat16 *g = static_cast<const __nv_bfloat16 *>(grad);
+        if (vec) {
+            unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count);
+            fold_vec_kernel<__nv_bfloat16, U><<<grid, kThreads, 0, stream>>>(g, m, v, n4, n, c.a,
+                                                                              c.b);
+        } else {
+            unsigned grid = grid_for(n, kThreads, sm_count);
+            fold_scalar_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>(g, m, v, n, c.a, c.b);
+        }
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants c, int sm_count,
+                         cudaStream_t stream) {
+    if (n == 0) return cudaSuccess;
+    constexpr int U = 4;
+    const size_t n4 = n / 4;
+    if (aligned(w, 16) && aligned(m, 16) && aligned(v, 16)) {
+        unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count, kApplyCtasPerSm);
+        apply_vec_kernel<U><<<grid, kThreads, 0, stream>>>(w, m, v, n4, n, c);
+    } else {
+        unsigned grid = grid_for(n, kThreads, sm_count);
+        apply_scalar_kernel<<<grid, kThreads, 0, stream>>>(w, m, v, n, c);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace adama

@@ -1,0 +1,532 @@
+// Fused linear-layer weight gradient + AdamA fold for sm_100a.
+//
+//   G[p,q]  = sum_tau X[tau,p] * dY[tau,q]          (bf16 x bf16 -> fp32, tcgen05.mma)
+//   m[p,q] += a*G[p,q];   v[p,q] += b*G[p,q]^2       (Algorithm 2, inner loop body)
+//
+// G lives only as an accumulator tile in tensor memory: the epilogue reads it with
+// tcgen05.ld, scales it, stages a*G and b*G^2 in shared memory and hands them to
+// the TMA unit as reduce-add stores, so m and v are read-modified-written at the
+// L2 and the SM never waits on a global load.
+//
+// Persistent kernel, one CTA per SM, 192 threads:
+//   warp 0      TMA producer: X and dY tiles -> 4-stage shared-memory ring
+//   warp 1      MMA issuer (single thread) + owner of the 512 TMEM columns
+//   warps 2..5  epilogue, one TMEM lane quarter each
+// The 512 TMEM columns hold two 128x256 fp32 accumulators, so the epilogue of tile
+// i overlaps the main loop of tile i+1.
+//
+// Operand layout.  The contraction runs over tokens, the strided dimension of both
+// row-major inputs, so both operands are "MN-major": a TMA box of 64 features x 64
+// tokens lands as 64 rows of 128 bytes (one token per row) under the 128-byte
+// swizzle; a 128-row A tile is two such boxes, a 256-column B tile four.  The
+// shared-memory matrix descriptor states: 8-token groups 1024 bytes apart (stride
+// byte offset), 64-feature groups one box (8192 bytes) apart (leading byte offset).
+//
+// Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the kernel
+// records a code in the status block, all roles drain and leave, TMEM is freed.
+#include <cuda.h>
+
+#include "adama_internal.h"
+
+namespace adama {
+namespace {
+
+constexpr int BM = 128;     // tile rows    (d_in  direction) = UMMA M
+constexpr int BN = 256;     // tile columns (d_out direction) = UMMA N
+constexpr int BK = 64;      // tokens per pipeline stage
+constexpr int UMMA_K = 16;  // tokens per tcgen05.mma (bf16)
+constexpr int STAGES = 4;
+constexpr int GROUP = 64;                                // features per 128-byte swizzled row
+constexpr int BOX_BYTES = GROUP * BK * 2;                // 8192
+constexpr int A_STAGE_BYTES = (BM / GROUP) * BOX_BYTES;  // 16384
+constexpr int B_STAGE_BYTES = (BN / GROUP) * BOX_BYTES;  // 32768
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int EPI_COLS = 32;                            // fp32 columns per reduce box (128 B)
+constexpr int EPI_ROWS = 32;                            // one TMEM lane quarter
+constexpr int EPI_BUF_BYTES = EPI_ROWS * EPI_COLS * 4;  // 4096
+constexpr int EPI_WARPS = 4;
+constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
+constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
+constexpr int TMEM_COLS = 512;
+constexpr int ACC_STAGES = 2;
+
+constexpr int SMEM_RING_OFF = 0;
+constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
+constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
+constexpr int SMEM_BAR_BYTES = 256;
+constexpr int SMEM_BYTES = SMEM_BAR_OFF + SMEM_BAR_BYTES + 1024;  // + slack for 1024-B alignment
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr unsigned long long kDrainLimitNs = 20000000ull;   // 20 ms
+
+// tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both
+// MN-major, N = 256, M = 128.
+constexpr uint32_t kInstrDesc = (1u << 4)      // D format: f32
+                                | (1u << 7)    // A format: bf16
+                                | (1u << 10)   // B format: bf16
+                                | (1u << 15)   // A is MN-major
+                                | (1u << 16)   // B is MN-major
+                                | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// ---- PTX wrappers --------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if `limit_ns` passed or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer();
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 0x3f) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer() - t0 > limit_ns) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int x, int y,
+                                                  uint32_t src) {
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group "
+        "[%0, {%1, %2}], [%3];" ::"l"(map),
+        "r"(x), "r"(y), "r"(src)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                     bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b,
+                                       uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i receives TMEM lane (base lane + i).
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
+          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, float x, float y, float z, float w) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z),
+                 "f"(w)
+                 : "memory");
+}
+
+// Shared-memory matrix descriptor for an MN-major bf16 operand under the 128-byte
+// swizzle: start address, leading byte offset (between 64-feature groups), stride
+// byte offset (between 8-token groups), descriptor version 1, layout SWIZZLE_128B.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+    constexpr uint64_t lbo = BOX_BYTES >> 4;  // 8192 B
+    constexpr uint64_t sbo = 1024 >> 4;       // 8 tokens x 128 B
+    return (uint64_t)((addr & 0x3ffff) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+
+struct Barriers {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t acc_full[ACC_STAGES];
+    uint64_t acc_empty[ACC_STAGES];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+static_assert(sizeof(Barriers) <= SMEM_BAR_BYTES, "barrier block");
+
+__device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars, unsigned site,
+                                               unsigned tile) {
+    *reinterpret_cast<volatile int *>(&bars->abort_flag) = 1;
+    if (atomicCAS(status, (unsigned)kDevOk, (unsigned)kDevTimeout) == kDevOk) {
+        status[1] = site;
+        status[2] = tile;
+    }
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
+                  const __grid_constant__ CUtensorMap map_dy,
+                  const __grid_constant__ CUtensorMap map_m,
+                  const __grid_constant__ CUtensorMap map_v, int tokens, int d_in, int d_out,
+                  float a, float b, unsigned *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;  // swizzled tiles need 1024-B alignment
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    Barriers *bars = reinterpret_cast<Barriers *>(smem + SMEM_BAR_OFF);
+    volatile int *abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int tiles_m = (d_in + BM - 1) / BM;
+    const int tiles_n = (d_out + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int num_kb = (tokens + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&bars->full[s]), 1);
+            mbar_init(smem_u32(&bars->empty[s]), 1);
+        }
+        for (int s = 0; s < ACC_STAGES; ++s) {
+            mbar_init(smem_u32(&bars->acc_full[s]), 1);
+            mbar_init(smem_u32(&bars->acc_empty[s]), EPI_WARPS);
+        }
+        mbar_init(smem_u32(&bars->drain), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&bars->tmem_base)),
+                     "n"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t armed = 0;        // bit s: stage s has been armed at least once
+        uint32_t last_parity = 0;  // bit s: parity of the phase last armed on stage s
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int m0 = (tile % tiles_m) * BM;
+            const int n0 = (tile / tiles_m) * BN;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) {
+                    if (lane == 0) record_timeout(status, bars, 1, (unsigned)tile);
+                    break;
+                }
+                if (lane == 0) {
+                    const uint32_t bar = smem_u32(&bars->full[stage]);
+                    const uint32_t sa = base + SMEM_RING_OFF + stage * STAGE_BYTES;
+                    const uint32_t sb = sa + A_STAGE_BYTES;
+                    // out-of-range parts of a box are zero-filled and still counted
+                    mbar_arrive_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+                    for (int j = 0; j < BM / GROUP; ++j)
+                        tma_load_2d(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK, bar);
+#pragma unroll
+                    for (int j = 0; j < BN / GROUP; ++j)
+                        tma_load_2d(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK, bar);
+                }
+                armed |= 1u << stage;
+                last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
+                __syncwarp();
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1;
+                }
+            }
+        }
+        if (*abort_flag) {
+            // leave no copy in flight behind: wait (bounded) for every armed stage to land
+            int never = 0;
+            for (int s = 0; s < STAGES; ++s)
+                if (armed & (1u << s))
+                    mbar_wait(smem_u32(&bars->full[s]), (last_parity >> s) & 1u, &never,
+                              kDrainLimitNs);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+            const int as = it & 1;
+            const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+            ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) record_timeout(status, bars, 2, (unsigned)tile);
+                break;
+            }
+            tc_fence_after();
+            const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
+            for (int kb = 0; kb < num_kb; ++kb) {
+                ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) {
+                    if (lane == 0) record_timeout(status, bars, 3, (unsigned)tile);
+                    break;
+                }
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t sa = base + SMEM_RING_OFF + stage * STAGE_BYTES;
+                    const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // 16 tokens further = 16 rows of 128 bytes
+                        const uint64_t da = make_smem_desc(sa + k * (UMMA_K * 128));
+                        const uint64_t db = make_smem_desc(sb + k * (UMMA_K * 128));
+                        tc_mma(tmem_d, da, db, kInstrDesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&bars->empty[stage]));  // stage free once these MMAs retire
+                }
+                __syncwarp();
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1;
+                }
+            }
+            if (ok && lane == 0) tc_commit(smem_u32(&bars->acc_full[as]));
+            __syncwarp();
+        }
+        if (*abort_flag) {
+            // let issued MMAs retire before TMEM is given back
+            if (lane == 0) tc_commit(smem_u32(&bars->drain));
+            __syncwarp();
+            int never = 0;
+            mbar_wait(smem_u32(&bars->drain), 0, &never, kDrainLimitNs);
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> a*G, b*G^2 -> TMA reduce-add into m, v ----------
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const uint32_t sm_m = base + SMEM_EPI_OFF + (uint32_t)q * 2 * EPI_BUF_BYTES;
+        const uint32_t sm_v = sm_m + EPI_BUF_BYTES;
+        // 128-byte swizzle: 16-byte chunk j of row r sits at chunk (j ^ (r & 7))
+        const uint32_t row_off = (uint32_t)lane * 128u;
+        const uint32_t sw = (uint32_t)(lane & 7);
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+            const int as = it & 1;
+            const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+            const int row0 = (tile % tiles_m) * BM + q * EPI_ROWS;
+            const int n0 = (tile / tiles_m) * BN;
+            ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) record_timeout(status, bars, 4, (unsigned)tile);
+                break;
+            }
+            tc_fence_after();
+            if (row0 < d_in) {
+                const uint32_t taddr0 =
+                    tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
+                for (int c = 0; c < BN / EPI_COLS; ++c) {
+                    const int col0 = n0 + c * EPI_COLS;
+                    if (col0 >= d_out) break;  // boxes wholly outside the matrix are skipped
+                    uint32_t r[32];
+                    tc_ld_32x32(taddr0 + (uint32_t)(c * EPI_COLS), r);
+                    tc_wait_ld();
+                    // first-moment increments
+                    if (lane == 0) bulk_wait_read<1>();  // previous reduce from the m buffer was read
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t addr = sm_m + row_off + ((((uint32_t)j) ^ sw) << 4);
+                        st_shared_v4(addr, a * __uint_as_float(r[4 * j + 0]),
+                                     a * __uint_as_float(r[4 * j + 1]),
+                                     a * __uint_as_float(r[4 * j + 2]),
+                                     a * __uint_as_float(r[4 * j + 3]));
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_reduce_add_2d(&map_m, col0, row0, sm_m);
+                        bulk_commit();
+                        bulk_wait_read<1>();  // previous reduce from the v buffer was read
+                    }
+                    __syncwarp();
+                    // second-moment increments
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t addr = sm_v + row_off + ((((uint32_t)j) ^ sw) << 4);
+                        const float g0 = __uint_as_float(r[4 * j + 0]);
+                        const float g1 = __uint_as_float(r[4 * j + 1]);
+                        const float g2 = __uint_as_float(r[4 * j + 2]);
+                        const float g3 = __uint_as_float(r[4 * j + 3]);
+                        st_shared_v4(addr, (b * g0) * g0, (b * g1) * g1, (b * g2) * g2,
+                                     (b * g3) * g3);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_reduce_add_2d(&map_v, col0, row0, sm_v);
+                        bulk_commit();
+                    }
+                }
+            }
+            // accumulator stage may now be overwritten by the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[as]));
+        }
+        if (lane == 0) bulk_wait_all();  // reduce-adds complete before the CTA retires
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "n"(TMEM_COLS)
+                     : "memory");
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+bool g_attr_set = false;
+
+// 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
+bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void *ptr,
+               uint64_t cols, uint64_t rows, uint64_t ld, uint32_t box_cols, uint32_t box_rows,
+               CUtensorMapL2promotion promo) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * elem};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t wgrad_fold_setup(const char **msg) {
+    if (!g_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000,
+                                                         cudaEnableDefault, &qres);
+        if (e != cudaSuccess) {
+            *msg = "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)";
+            return e;
+        }
+        if (qres != cudaDriverEntryPointSuccess || !fn) {
+            *msg = "driver has no cuTensorMapEncodeTiled";
+            return cudaErrorNotSupported;
+        }
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
+    cudaError_t e = wgrad_fold_setup(msg);
+    if (e != cudaSuccess) return e;
+    if (!g_attr_set) {
+        e = cudaFuncSetAttribute(wgrad_fold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SMEM_BYTES);
+        if (e != cudaSuccess) {
+            *msg = "cudaFuncSetAttribute(wgrad_fold_kernel)";
+            return e;
+        }
+        g_attr_set = true;
+    }
+    CUtensorMap map_x, map_dy, map_m, map_v;
+    bool ok = encode_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.X, (uint64_t)p.d_in,
+                        (uint64_t)p.tokens, (uint64_t)p.ldx, GROUP, BK,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B) &&
+              encode_2d(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.dY, (uint64_t)p.d_out,
+                        (uint64_t)p.tokens, (uint64_t)p.ldy, GROUP, BK,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B) &&
+              encode_2d(&map_m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.m, (uint64_t)p.d_out,
+                        (uint64_t)p.d_in, (uint64_t)p.ldmv, EPI_COLS, EPI_ROWS,
+                        CU_TENSOR_MAP_L2_PROMOTION_NONE) &&
+              encode_2d(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.v, (uint64_t)p.d_out,
+                        (uint64_t)p.d_in, (uint64_t)p.ldmv, EPI_COLS, EPI_ROWS,
+                        CU_TENSOR_MAP_L2_PROMOTION_NONE);
+    if (!ok) {
+        *msg = "cuTensorMapEncodeTiled rejected a tensor";
+        return cudaErrorInvalidValue;
+    }
+    const int tiles = ((p.d_in + BM - 1) / BM) * ((p.d_out + BN - 1) / BN);
+    const int grid = tiles < p.sm_count ? tiles : p.sm_count;
+    wgrad_fold_kernel<<<grid, NUM_THREADS, SMEM_BYTES, p.stream>>>(
+        map_x, map_dy, map_m, map_v, p.tokens, p.d_in, p.d_out, p.c.a, p.c.b, p.status);
+    *msg = "wgrad_fold launch";
+    return cudaGetLastError();
+}
+
+}  // namespace adama
