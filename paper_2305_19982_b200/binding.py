@@ -1,0 +1,274 @@
+"""ctypes binding with the same names as the C ABI (include/adama.h).
+
+Argument marshalling only: tensors become raw device pointers, the stream is
+torch's current CUDA stream, doubles stay doubles.
+"""
+from __future__ import annotations
+
+import ctypes
+import enum
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libadama.so"
+
+EXPORTED_SYMBOLS = [
+    "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_fold_host", "adama_linear_wgrad_fold_host",
+    "adama_apply_to_host", "adama_get_step", "adama_set_step", "adama_get_n_micro",
+    "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
+    "adama_version",
+]
+
+
+class Status(enum.IntEnum):
+    OK = 0
+    ERR_INVALID_ARG = 1
+    ERR_BAD_STATE = 2
+    ERR_MISALIGNED = 3
+    ERR_UNSUPPORTED = 4
+    ERR_CUDA = 5
+    ERR_TIMEOUT = 6
+
+
+F32, BF16 = 0, 1
+GRADS_PRESCALED = 1
+
+
+class AdamAError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        self.status = Status(status)
+        super().__init__(f"{self.status.name}: {message}")
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("beta1", ctypes.c_double), ("beta2", ctypes.c_double), ("eps", ctypes.c_double),
+                ("device", ctypes.c_int), ("flags", ctypes.c_uint)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libadama.so (built in-tree by paper_2305_19982_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise FileNotFoundError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2305_19982_b200.build` "
+            "(there is no fallback path)")
+    L = ctypes.CDLL(str(_LIB_PATH))
+    vp, i64, sz, dbl, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_double, ctypes.c_int
+    L.adama_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_Config)]
+    L.adama_destroy.argtypes = [vp]
+    L.adama_begin_minibatch.argtypes = [vp, ci]
+    L.adama_fold.argtypes = [vp, vp, ci, vp, vp, sz, vp]
+    L.adama_linear_wgrad_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp]
+    L.adama_apply.argtypes = [vp, vp, vp, vp, sz, dbl, vp]
+    L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
+    L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
+    L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
+    L.adama_get_step.argtypes = [vp]
+    L.adama_get_step.restype = i64
+    L.adama_set_step.argtypes = [vp, i64]
+    L.adama_get_n_micro.argtypes = [vp]
+    L.adama_sync_status.argtypes = [vp, vp]
+    L.adama_last_error.argtypes = [vp]
+    L.adama_last_error.restype = ctypes.c_char_p
+    L.adama_launch_count.argtypes = [vp]
+    L.adama_launch_count.restype = i64
+    L.adama_host_constants.argtypes = [ctypes.POINTER(_Config), ci, i64, dbl,
+                                       ctypes.POINTER(ctypes.c_float)]
+    L.adama_version.restype = ctypes.c_char_p
+    _lib = L
+    return L
+
+
+def host_constants(beta1, beta2, eps, n_micro, t, lr, flags=0):
+    """adama_host_constants: the nine fp32 constants the kernels receive (no GPU needed)."""
+    L = load_library()
+    cfg = _Config(beta1, beta2, eps, 0, flags)
+    out = (ctypes.c_float * 9)()
+    st = L.adama_host_constants(ctypes.byref(cfg), n_micro, t, lr, out)
+    if st != 0:
+        raise AdamAError(st, "adama_host_constants")
+    return [float(x) for x in out]
+
+
+def _stream_ptr(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _dev_ptr(t: torch.Tensor, dtype: torch.dtype, name: str) -> int:
+    if not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+class AdamA:
+    """One AdamA context (adama_ctx) bound to a CUDA device.
+
+    Methods mirror the C ABI one to one; tensors are torch CUDA tensors owned by
+    the caller, work is queued on torch's current stream of the context's device.
+    """
+
+    def __init__(self, beta1=0.9, beta2=0.999, eps=1e-8, device=0, grads_prescaled=False):
+        self._L = load_library()
+        self._h = ctypes.c_void_p()
+        self.device = torch.device("cuda", int(device))
+        cfg = _Config(beta1, beta2, eps, int(device), GRADS_PRESCALED if grads_prescaled else 0)
+        st = self._L.adama_init(ctypes.byref(self._h), ctypes.byref(cfg))
+        if st != 0:
+            self._h = ctypes.c_void_p()
+            raise AdamAError(st, "adama_init failed (needs a compute-capability-10.x GPU)")
+
+    # -- plumbing ---------------------------------------------------------------------------
+    def _check(self, st: int) -> None:
+        if st != 0:
+            raise AdamAError(st, self._L.adama_last_error(self._h).decode())
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._L.adama_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- Algorithm 2 --------------------------------------------------------------------------
+    def begin_minibatch(self, n_micro: int) -> None:
+        self._check(self._L.adama_begin_minibatch(self._h, int(n_micro)))
+
+    def fold(self, grad: torch.Tensor, m: torch.Tensor, v: torch.Tensor) -> None:
+        """adama_fold on contiguous tensors of equal numel; grad is fp32 or bf16."""
+        if grad.dtype == torch.float32:
+            gdt = F32
+        elif grad.dtype == torch.bfloat16:
+            gdt = BF16
+        else:
+            raise TypeError("grad must be float32 or bfloat16")
+        if not (grad.is_contiguous() and m.is_contiguous() and v.is_contiguous()):
+            raise ValueError("fold needs contiguous tensors")
+        n = grad.numel()
+        if m.numel() != n or v.numel() != n:
+            raise ValueError("grad, m, v must have the same number of elements")
+        self._check(self._L.adama_fold(self._h, _dev_ptr(grad, grad.dtype, "grad"), gdt,
+                                       _dev_ptr(m, torch.float32, "m"),
+                                       _dev_ptr(v, torch.float32, "v"), n,
+                                       _stream_ptr(self.device)))
+
+    def linear_wgrad_fold(self, X: torch.Tensor, dY: torch.Tensor, m: torch.Tensor,
+                          v: torch.Tensor) -> None:
+        """adama_linear_wgrad_fold: X [tokens, d_in], dY [tokens, d_out] bf16 (unit stride in
+        the last dim), m, v [d_in, d_out] fp32 views with a common row pitch."""
+        if X.dim() != 2 or dY.dim() != 2 or m.dim() != 2 or v.dim() != 2:
+            raise ValueError("linear_wgrad_fold takes 2-D tensors")
+        tokens, d_in = X.shape
+        if dY.shape[0] != tokens:
+            raise ValueError("X and dY must have the same number of tokens")
+        d_out = dY.shape[1]
+        if tuple(m.shape) != (d_in, d_out) or tuple(v.shape) != (d_in, d_out):
+            raise ValueError("m, v must be [d_in, d_out]")
+        for name, t in (("X", X), ("dY", dY), ("m", m), ("v", v)):
+            if t.shape[1] > 1 and t.stride(1) != 1:
+                raise ValueError(f"{name} must have unit stride in its last dimension")
+        if m.stride(0) != v.stride(0):
+            raise ValueError("m and v must share one row pitch")
+        ldx = X.stride(0) if tokens > 1 else max(d_in, X.stride(0))
+        ldy = dY.stride(0) if tokens > 1 else max(d_out, dY.stride(0))
+        ldmv = m.stride(0) if d_in > 1 else max(d_out, m.stride(0))
+        self._check(self._L.adama_linear_wgrad_fold(
+            self._h, _dev_ptr(X, torch.bfloat16, "X"), _dev_ptr(dY, torch.bfloat16, "dY"),
+            tokens, d_in, d_out, ldx, ldy, _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), ldmv, _stream_ptr(self.device)))
+
+    def apply(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float) -> None:
+        if not (w.is_contiguous() and m.is_contiguous() and v.is_contiguous()):
+            raise ValueError("apply needs contiguous tensors")
+        n = w.numel()
+        if m.numel() != n or v.numel() != n:
+            raise ValueError("w, m, v must have the same number of elements")
+        self._check(self._L.adama_apply(self._h, _dev_ptr(w, torch.float32, "w"),
+                                        _dev_ptr(m, torch.float32, "m"),
+                                        _dev_ptr(v, torch.float32, "v"), n, float(lr),
+                                        _stream_ptr(self.device)))
+
+    # -- host-buffer variants ---------------------------------------------------------------
+    def fold_host(self, grad_host: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
+                  staging: torch.Tensor) -> None:
+        if grad_host.is_cuda or not grad_host.is_contiguous():
+            raise TypeError("grad_host must be a contiguous CPU tensor (pinned for full speed)")
+        gdt = {torch.float32: F32, torch.bfloat16: BF16}[grad_host.dtype]
+        n = grad_host.numel()
+        if m.numel() != n or v.numel() != n:
+            raise ValueError("grad, m, v must have the same number of elements")
+        self._check(self._L.adama_fold_host(
+            self._h, grad_host.data_ptr(), gdt, _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), n, staging.data_ptr(),
+            staging.numel() * staging.element_size(), _stream_ptr(self.device)))
+
+    def linear_wgrad_fold_host(self, X_host: torch.Tensor, dY_host: torch.Tensor, m: torch.Tensor,
+                               v: torch.Tensor, staging: torch.Tensor) -> None:
+        if X_host.is_cuda or dY_host.is_cuda:
+            raise TypeError("X_host, dY_host must be CPU tensors")
+        if not (X_host.is_contiguous() and dY_host.is_contiguous()):
+            raise ValueError("X_host, dY_host must be dense")
+        if X_host.dtype != torch.bfloat16 or dY_host.dtype != torch.bfloat16:
+            raise TypeError("X_host, dY_host must be bfloat16")
+        tokens, d_in = X_host.shape
+        d_out = dY_host.shape[1]
+        if tuple(m.shape) != (d_in, d_out) or tuple(v.shape) != (d_in, d_out):
+            raise ValueError("m, v must be [d_in, d_out]")
+        self._check(self._L.adama_linear_wgrad_fold_host(
+            self._h, X_host.data_ptr(), dY_host.data_ptr(), tokens, d_in, d_out,
+            _dev_ptr(m, torch.float32, "m"), _dev_ptr(v, torch.float32, "v"), m.stride(0),
+            staging.data_ptr(), staging.numel() * staging.element_size(),
+            _stream_ptr(self.device)))
+
+    def apply_to_host(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float,
+                      w_host: torch.Tensor) -> None:
+        n = w.numel()
+        if w_host.is_cuda or w_host.dtype != torch.float32 or w_host.numel() != n:
+            raise TypeError("w_host must be a CPU float32 tensor of w's size")
+        self._check(self._L.adama_apply_to_host(
+            self._h, _dev_ptr(w, torch.float32, "w"), _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), n, float(lr), w_host.data_ptr(),
+            _stream_ptr(self.device)))
+
+    # -- state ------------------------------------------------------------------------------
+    @property
+    def step(self) -> int:
+        return int(self._L.adama_get_step(self._h))
+
+    def set_step(self, t: int) -> None:
+        self._check(self._L.adama_set_step(self._h, int(t)))
+
+    @property
+    def n_micro(self) -> int:
+        return int(self._L.adama_get_n_micro(self._h))
+
+    def sync_status(self) -> None:
+        """Waits for the current stream and raises AdamAError(ERR_TIMEOUT) if a bounded
+        device-side wait expired."""
+        self._check(self._L.adama_sync_status(self._h, _stream_ptr(self.device)))
+
+    @property
+    def launch_count(self) -> int:
+        return int(self._L.adama_launch_count(self._h))
+
+
+def version() -> str:
+    return load_library().adama_version().decode()

@@ -1,0 +1,249 @@
+"""GPU parity of the fused weight-gradient + fold kernel against the fp64 oracle.
+
+The oracle forms G = X^T.dY by the naive triple loop (or entry by entry for sampled
+checks) and folds it as Algorithm 2 states.  Tolerance for the bf16-input path: relative
+L2 error <= 2e-3 on m, v and w; with small-integer inputs the fp32 accumulation is exact
+and the fp32 fold tolerance (1e-6) applies.
+"""
+import numpy as np
+import pytest
+import torch
+
+import adama_workloads as wl
+import oracle
+import paper_2305_19982_b200 as adama
+from oracle import AdamAOracle
+from parity import SENTINEL, f64, rel_l2
+
+pytestmark = pytest.mark.gpu
+TOL_BF16 = 2e-3
+TOL_EXACT = 1e-6
+
+
+def _draw(T, d_in, d_out, seed, integer=False):
+    if integer:
+        X = wl.small_integers((T, d_in), 4, torch.bfloat16, seed)
+        dY = wl.small_integers((T, d_out), 4, torch.bfloat16, seed + 1)
+    else:
+        X = wl.normal((T, d_in), 1.0, torch.bfloat16, seed)
+        dY = wl.normal((T, d_out), 1e-2, torch.bfloat16, seed + 1)
+    return X, dY
+
+
+def _full_parity(T, d_in, d_out, n_micro=2, steps=1, integer=False, pad=0, tol=None):
+    """Whole-matrix comparison; `pad` > 0 embeds X, dY, m, v in wider buffers (row pitch >
+    row length) whose extra columns hold a sentinel that must survive."""
+    tol = tol if tol is not None else (TOL_EXACT if integer else TOL_BF16)
+    opt = adama.AdamA()
+    w0 = wl.normal((d_in, d_out), 0.02, torch.float32, 77)
+    orc = AdamAOracle(f64(w0))
+    pad_mv = pad and ((pad + 3) // 4) * 4
+    pad_in = pad and ((pad + 7) // 8) * 8
+    mbuf = torch.full((d_in, d_out + pad_mv), SENTINEL, device="cuda")
+    vbuf = torch.full((d_in, d_out + pad_mv), SENTINEL, device="cuda")
+    m, v = mbuf[:, :d_out], vbuf[:, :d_out]
+    m.zero_()
+    v.zero_()
+    w = w0.cuda()
+    for step in range(steps):
+        opt.begin_minibatch(n_micro)
+        orc.begin_minibatch(n_micro)
+        for i in range(n_micro):
+            X, dY = _draw(T, d_in, d_out, 1000 * step + 10 * i + d_in, integer)
+            Xb = torch.full((T, d_in + pad_in), 7.0, dtype=torch.bfloat16, device="cuda")
+            Yb = torch.full((T, d_out + pad_in), 7.0, dtype=torch.bfloat16, device="cuda")
+            Xb[:, :d_in] = X.cuda()
+            Yb[:, :d_out] = dY.cuda()
+            opt.linear_wgrad_fold(Xb[:, :d_in], Yb[:, :d_out], m, v)
+            orc.fold_linear(f64(X), f64(dY))
+        opt.sync_status()
+        assert rel_l2(f64(m), orc.m) <= tol
+        assert rel_l2(f64(v), orc.v) <= tol
+        # apply works on contiguous buffers: use dense copies of the views
+        mc, vc = m.contiguous(), v.contiguous()
+        opt.apply(w, mc, vc, wl.LR)
+        orc.update(wl.LR)
+        m.copy_(mc)
+        v.copy_(vc)
+        assert rel_l2(f64(w), orc.theta) <= tol
+    if pad:
+        assert bool((mbuf[:, d_out:] == SENTINEL).all()) and bool((vbuf[:, d_out:] == SENTINEL).all())
+    opt.close()
+
+
+def test_single_tile_integer_inputs_exact():
+    _full_parity(64, 128, 256, integer=True)
+
+
+def test_single_tile_partial_k():
+    """tokens not a multiple of the 64-token stage nor of the 16-token MMA."""
+    _full_parity(100, 128, 256, integer=True)
+    _full_parity(7, 128, 256, integer=True)
+
+
+def test_operand_roles_not_swapped():
+    """d_in != d_out and one-hot activations: G is a scatter-add of dY rows, so a swapped or
+    transposed operand cannot pass."""
+    T, d_in, d_out = 96, 136, 264
+    idx = torch.randint(0, d_in, (T,), generator=torch.Generator().manual_seed(3))
+    X = torch.zeros(T, d_in, dtype=torch.bfloat16)
+    X[torch.arange(T), idx] = 1.0
+    dY = wl.small_integers((T, d_out), 8, torch.bfloat16, 5)
+    opt = adama.AdamA()
+    opt.begin_minibatch(1)
+    m = torch.zeros(d_in, d_out, device="cuda")
+    v = torch.zeros(d_in, d_out, device="cuda")
+    opt.linear_wgrad_fold(X.cuda(), dY.cuda(), m, v)
+    opt.sync_status()
+    G = np.zeros((d_in, d_out))
+    for tau in range(T):
+        G[idx[tau]] += f64(dY[tau])
+    np.testing.assert_allclose(f64(m), (1 - wl.BETA1) * G, rtol=1e-6, atol=1e-12)
+    np.testing.assert_allclose(f64(v), (1 - wl.BETA2) * G * G, rtol=1e-6, atol=1e-12)
+    opt.close()
+
+
+@pytest.mark.parametrize("T,d_in,d_out", [(100, 200, 328), (64, 8, 8), (130, 136, 520),
+                                          (33, 1, 8), (64, 129, 257 + 7)])
+def test_ragged_shapes(T, d_in, d_out):
+    """Shapes that are no multiple of the 128x256 tile, the 64-feature TMA box or the
+    32x32 reduce box; integer inputs make the contraction exact."""
+    if d_out % 8:
+        d_out += 8 - d_out % 8
+    _full_parity(T, d_in if d_in % 8 == 0 or d_in == 1 else d_in + 8 - d_in % 8, d_out,
+                 integer=True, pad=5)
+
+
+def test_multi_tile_normal_inputs_two_steps():
+    _full_parity(512, 384, 768, n_micro=2, steps=2)
+
+
+def test_more_tiles_than_sms():
+    """16 x 16 = 256 tiles on 148 SMs: persistent CTAs take a second tile and both
+    accumulator stages, with phase wrap-around of the 4-stage ring (T=640: 10 k-blocks)."""
+    _full_parity(640, 2048, 4096, n_micro=1, integer=False)
+
+
+def test_long_contraction_phase_wraps():
+    _full_parity(4096 + 48, 256, 512, n_micro=1)
+
+
+def _sampled_entries(d_in, d_out, count, seed):
+    rng = np.random.default_rng(seed)
+    p = rng.integers(0, d_in, count)
+    q = rng.integers(0, d_out, count)
+    # corners and the last rows / columns (ragged tiles) are always included
+    edge_p = [0, 0, d_in - 1, d_in - 1, d_in - 1, d_in // 2]
+    edge_q = [0, d_out - 1, 0, d_out - 1, d_out // 2, d_out - 1]
+    return np.concatenate([p, edge_p]), np.concatenate([q, edge_q])
+
+
+def _sampled_parity(T, d_in, d_out, n_micro, steps, config, count=3000):
+    """Benchmark-sized layers: sampled entries (each a T-term dot product in the oracle)
+    plus one whole 128x256 tile at the bottom-right corner."""
+    opt = adama.AdamA()
+    p, q = _sampled_entries(d_in, d_out, count, config)
+    r0, c0 = max(0, d_in - 128), max(0, d_out - 256)
+    tp, tq = np.meshgrid(np.arange(r0, d_in), np.arange(c0, d_out), indexing="ij")
+    p = np.concatenate([p, tp.reshape(-1)])
+    q = np.concatenate([q, tq.reshape(-1)])
+    flat = torch.from_numpy(p * d_out + q).cuda()
+    w = wl.normal((d_in, d_out), 0.02, torch.float32, wl.seed_for(config, 99), device="cuda")
+    m = torch.zeros(d_in, d_out, device="cuda")
+    v = torch.zeros(d_in, d_out, device="cuda")
+    orc = AdamAOracle(f64(w.view(-1)[flat]))
+    for step in range(steps):
+        opt.begin_minibatch(n_micro)
+        orc.begin_minibatch(n_micro)
+        for i in range(n_micro):
+            X = wl.normal((T, d_in), 1.0, torch.bfloat16, wl.seed_for(config, step, i), device="cuda")
+            dY = wl.normal((T, d_out), 1e-2, torch.bfloat16, wl.seed_for(config, step, i) + 50,
+                           device="cuda")
+            opt.linear_wgrad_fold(X, dY, m, v)
+            orc.fold(oracle.linear_wgrad_entries(f64(X), f64(dY), p, q))
+        opt.sync_status()
+        assert rel_l2(f64(m.view(-1)[flat]), orc.m) <= TOL_BF16
+        assert rel_l2(f64(v.view(-1)[flat]), orc.v) <= TOL_BF16
+        opt.apply(w, m, v, wl.LR)
+        orc.update(wl.LR)
+        assert rel_l2(f64(w.view(-1)[flat]), orc.theta) <= TOL_BF16
+        assert rel_l2(f64(m.view(-1)[flat]), wl.BETA1 * orc.m) <= TOL_BF16
+    assert bool((v >= 0).all()) and bool(torch.isfinite(m).all()) and bool(torch.isfinite(w).all())
+    opt.close()
+
+
+def test_config3_sampled():
+    """d_in = d_out = 4096, 4096 tokens, N=4, 3 steps (the benchmark's linear layer)."""
+    c = wl.CONFIG3
+    _sampled_parity(c.tokens, c.d_in, c.d_out, c.n_micro, c.steps, 3)
+
+
+@pytest.mark.parametrize("name,d_in,d_out", wl.gpt2xl_block_linears())
+def test_config4_layer_shapes_sampled(name, d_in, d_out):
+    """GPT-2-XL-shaped linears (1600 = 12.5 tiles of 128, 4800 = 18.75 tiles of 256)."""
+    _sampled_parity(wl.CONFIG4_TOKENS, d_in, d_out, 2, 1, 4, count=1500)
+
+
+@pytest.mark.parametrize("name,d_in,d_out", [x for x in wl.llama7b_block_linears()
+                                              if x[0] in ("gate", "down")])
+def test_config5_layer_shapes_sampled(name, d_in, d_out):
+    _sampled_parity(wl.CONFIG5_TOKENS, d_in, d_out, 1, 1, 5, count=1500)
+
+
+def test_zero_tokens_is_a_noop():
+    opt = adama.AdamA()
+    opt.begin_minibatch(1)
+    m = torch.ones(64, 64, device="cuda")
+    v = torch.ones(64, 64, device="cuda")
+    e = torch.empty(0, 64, dtype=torch.bfloat16, device="cuda")
+    before = opt.launch_count
+    opt.linear_wgrad_fold(e, e.clone(), m, v)
+    assert opt.launch_count == before and bool((m == 1).all())
+    opt.close()
+
+
+def test_run_twice_is_deterministic():
+    T, d_in, d_out = 256, 384, 512
+    X, dY = _draw(T, d_in, d_out, 11)
+    outs = []
+    for _ in range(2):
+        opt = adama.AdamA()
+        opt.begin_minibatch(3)
+        m = torch.zeros(d_in, d_out, device="cuda")
+        v = torch.zeros(d_in, d_out, device="cuda")
+        for _ in range(3):
+            opt.linear_wgrad_fold(X.cuda(), dY.cuda(), m, v)
+        opt.sync_status()
+        outs.append((m.clone(), v.clone()))
+        opt.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
+def test_host_buffer_variants_match_device_variants():
+    T, d_in, d_out, n = 128, 256, 512, 256 * 512
+    X, dY = _draw(T, d_in, d_out, 21)
+    g = wl.normal((n,), 1e-3, torch.bfloat16, 22)
+    res = []
+    for host in (False, True):
+        opt = adama.AdamA()
+        opt.begin_minibatch(2)
+        w = wl.normal((d_in, d_out), 0.02, torch.float32, 23).cuda()
+        m = torch.zeros(d_in, d_out, device="cuda")
+        v = torch.zeros(d_in, d_out, device="cuda")
+        if host:
+            staging = torch.empty(4 << 20, dtype=torch.uint8, device="cuda")
+            w_host = torch.empty(n, dtype=torch.float32).pin_memory()
+            opt.linear_wgrad_fold_host(X.pin_memory(), dY.pin_memory(), m, v, staging)
+            opt.fold_host(g.pin_memory(), m.view(-1), v.view(-1), staging)
+            opt.apply_to_host(w, m, v, wl.LR, w_host)
+            opt.sync_status()
+            assert torch.equal(w_host, w.cpu().view(-1))
+        else:
+            opt.linear_wgrad_fold(X.cuda(), dY.cuda(), m, v)
+            opt.fold(g.cuda(), m.view(-1), v.view(-1))
+            opt.apply(w, m, v, wl.LR)
+            opt.sync_status()
+        res.append((w.cpu(), m.cpu(), v.cpu()))
+        opt.close()
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
