@@ -1,0 +1,478 @@
+#!/usr/bin/env python
+"""Benchmark of the AdamA hot path on B200: fold / apply GB/s and fused wgrad+fold TFLOP/s.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload headline|gpt2xl|llama7b]
+
+One step of the headline workload = one pass of the whole path:
+  phase A  (flat 335M-parameter buffer, bf16 gradients, N=8):
+           begin_minibatch, 8 x fold, apply
+  phase B  (one 4096x4096 linear layer, 4096 tokens per micro-batch, N=4):
+           begin_minibatch, 4 x linear_wgrad_fold, apply
+All inputs are seeded synthetic tensors resident in HBM before the timed region.  Every
+fold reads 6 GB and every fused call touches 335 MB, far more than the 126 MB L2, so
+no L2 flush is needed between iterations.  Prints ONE JSON line.
+
+`--impl reference` times the fp64 CPU oracle (plain C, as it stands) on a bounded sample
+of the same workload on the host cores; it is a deliberately slow program, reported as a
+baseline only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import adama_workloads as wl  # noqa: E402
+
+METRIC = "adama_fold_apply_wgrad_algorithmic_GBps"
+UNIT = "GB/s"
+
+FOLD_BYTES_BF16 = 18   # 2 B gradient + 8 B read m,v + 8 B write m,v
+FOLD_BYTES_F32 = 20
+APPLY_BYTES = 24       # read + write of w, m, v
+
+
+def peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+def step_bytes_and_flops(n_flat, n_micro_flat, tokens, d_in, d_out, n_micro_lin):
+    """Algorithmic bytes and tensor flops of one headline step."""
+    flat = n_flat * (FOLD_BYTES_BF16 * n_micro_flat + APPLY_BYTES)
+    lin_params = d_in * d_out
+    lin_call = 16 * lin_params + 2 * tokens * (d_in + d_out)
+    lin = n_micro_lin * lin_call + APPLY_BYTES * lin_params
+    flops = n_micro_lin * 2.0 * tokens * d_in * d_out
+    return flat, lin, flops, lin_call
+
+
+# ---- clocks ------------------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) != 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+# ---- the CPU oracle arm ------------------------------------------------------------------------
+
+def oracle_sample_step(state):
+    """One bounded sample of the headline step in the fp64 oracle (same flow, smaller sizes)."""
+    import numpy as np
+    import oracle
+    flat, lin, grads, xs, ys = state["flat"], state["lin"], state["grads"], state["xs"], state["ys"]
+    flat.begin_minibatch(len(grads))
+    for g in grads:
+        flat.fold(g)
+    flat.update(wl.LR)
+    lin.begin_minibatch(len(xs))
+    for X, dY in zip(xs, ys):
+        lin.fold(oracle.linear_wgrad(X, dY).reshape(-1))
+    lin.update(wl.LR)
+    return np  # keep numpy imported
+
+
+def make_oracle_state(n_flat, tokens, d_in, d_out):
+    import numpy as np
+    import oracle
+    from oracle import AdamAOracle
+    f64 = lambda t: t.to(torch.float64).numpy()
+    flat = AdamAOracle(f64(wl.normal((n_flat,), 0.02, torch.float32, wl.seed_for(2, 99))))
+    grads = [f64(wl.normal((n_flat,), wl.CONFIG2.grad_std, torch.bfloat16, wl.seed_for(2, 0, i)))
+             for i in range(wl.CONFIG2.n_micro)]
+    lin = AdamAOracle(f64(wl.normal((d_in * d_out,), 0.02, torch.float32, wl.seed_for(3, 99))))
+    xs = [f64(wl.normal((tokens, d_in), 1.0, torch.bfloat16, wl.seed_for(3, 0, i)))
+          for i in range(wl.CONFIG3.n_micro)]
+    ys = [f64(wl.normal((tokens, d_out), 1e-2, torch.bfloat16, wl.seed_for(3, 0, i) + 50))
+          for i in range(wl.CONFIG3.n_micro)]
+    return {"flat": flat, "lin": lin, "grads": grads, "xs": xs, "ys": ys,
+            "threads": oracle.num_threads()}
+
+
+def time_oracle(n_flat, tokens, d_in, d_out, steps, warmup):
+    state = make_oracle_state(n_flat, tokens, d_in, d_out)
+    for _ in range(warmup):
+        oracle_sample_step(state)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample_step(state)
+    dt = (time.perf_counter() - t0) / steps
+    flat_b, lin_b, flops, _ = step_bytes_and_flops(n_flat, wl.CONFIG2.n_micro, tokens, d_in, d_out,
+                                                   wl.CONFIG3.n_micro)
+    sample = (f"flat buffer of {n_flat} params (of {wl.CONFIG2_FULL_N}), N=8 bf16-valued grads; "
+              f"linear layer {d_in}x{d_out}, {tokens} tokens (of 4096x4096, 4096), N=4; "
+              "same flow, fp64, OpenMP over elements")
+    return {"value": (flat_b + lin_b) / dt / 1e9, "unit": UNIT, "cores": state["threads"],
+            "kind": "oracle", "sample": sample, "seconds_per_sample_step": dt,
+            "wgrad_gflops": flops / dt / 1e9}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    base = time_oracle(1 << 24, 256, 512, 512, args.steps, args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": base["seconds_per_sample_step"] * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "headline (bounded sample per step): " + base["sample"]},
+            "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- our arm -----------------------------------------------------------------------------------
+
+class EventTimer:
+    """CUDA events recorded on torch's current stream (the stream every launch goes to)."""
+
+    def __init__(self):
+        self.marks = []
+
+    def mark(self, label):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        self.marks.append((label, ev))
+
+    def durations(self):
+        """label -> list of ms between a mark and the next mark."""
+        out = {}
+        for (label, ev), (_, nxt) in zip(self.marks[:-1], self.marks[1:]):
+            if label is not None:
+                out.setdefault(label, []).append(ev.elapsed_time(nxt))
+        return out
+
+
+def run_ours(args):
+    import paper_2305_19982_b200 as adama
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    pk = peaks()
+
+    n = args.flat_params
+    NA, NB = wl.CONFIG2.n_micro, wl.CONFIG3.n_micro
+    T, d_in, d_out = wl.CONFIG3.tokens, wl.CONFIG3.d_in, wl.CONFIG3.d_out
+    seed_shift = 100000 * rank  # each rank owns its own replica's data (weak scaling)
+
+    # phase A state and inputs
+    optA = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=local)
+    w = wl.normal((n,), 0.02, torch.float32, wl.seed_for(2, 99) + seed_shift, device=dev)
+    m = torch.zeros(n, device=dev)
+    v = torch.zeros(n, device=dev)
+    grads = [wl.normal((n,), wl.CONFIG2.grad_std, torch.bfloat16, wl.seed_for(2, 0, i) + seed_shift,
+                       device=dev) for i in range(NA)]
+    # phase B state and inputs
+    optB = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=local)
+    wB = wl.normal((d_in, d_out), 0.02, torch.float32, wl.seed_for(3, 99) + seed_shift, device=dev)
+    mB = torch.zeros(d_in, d_out, device=dev)
+    vB = torch.zeros(d_in, d_out, device=dev)
+    Xs = [wl.normal((T, d_in), 1.0, torch.bfloat16, wl.seed_for(3, 0, i) + seed_shift, device=dev)
+          for i in range(NB)]
+    dYs = [wl.normal((T, d_out), 1e-2, torch.bfloat16, wl.seed_for(3, 0, i) + 50 + seed_shift,
+                     device=dev) for i in range(NB)]
+
+    def step(timer=None):
+        mark = timer.mark if timer else (lambda label: None)
+        optA.begin_minibatch(NA)
+        for i in range(NA):
+            mark("fold")
+            optA.fold(grads[i], m, v)
+        mark("apply")
+        optA.apply(w, m, v, wl.LR)
+        optB.begin_minibatch(NB)
+        for i in range(NB):
+            mark("wgrad_fold")
+            optB.linear_wgrad_fold(Xs[i], dYs[i], mB, vB)
+        mark("apply_linear")
+        optB.apply(wB, mB, vB, wl.LR)
+        mark(None)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches0 = optA.launch_count + optB.launch_count
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    time.sleep(0.25)
+    timer = EventTimer()
+    barrier()
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step(timer)
+    stop.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(stop)
+    launches = optA.launch_count + optB.launch_count - launches0
+    optA.sync_status()
+    optB.sync_status()
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    flat_b, lin_b, flops, lin_call_b = step_bytes_and_flops(n, NA, T, d_in, d_out, NB)
+    value = world * (flat_b + lin_b) / (ms_per_step * 1e-3) / 1e9
+
+    dur = timer.durations()
+    avg = {k: sum(x) / len(x) for k, x in dur.items()}
+    fold_gbs = FOLD_BYTES_BF16 * n / (avg["fold"] * 1e-3) / 1e9
+    apply_gbs = APPLY_BYTES * n / (avg["apply"] * 1e-3) / 1e9
+    wgrad_tf = 2.0 * T * d_in * d_out / (avg["wgrad_fold"] * 1e-3) / 1e12
+    roof_kernels = {
+        "fold_bf16": {"bound": "hbm", "achieved": fold_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                      "frac": fold_gbs / pk["hbm_gbs"], "ms": avg["fold"],
+                      "bytes_per_param": FOLD_BYTES_BF16, "params": n},
+        "apply": {"bound": "hbm", "achieved": apply_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                  "frac": apply_gbs / pk["hbm_gbs"], "ms": avg["apply"],
+                  "bytes_per_param": APPLY_BYTES, "params": n},
+        "wgrad_fold": {"bound": "tensor", "achieved": wgrad_tf, "peak": pk["bf16_tflops"],
+                       "unit": "TFLOP/s", "frac": wgrad_tf / pk["bf16_tflops"],
+                       "frac_of_sustained": wgrad_tf / pk["bf16_tflops_sustained"],
+                       "ms": avg["wgrad_fold"], "flops_per_call": 2.0 * T * d_in * d_out,
+                       "hbm_bytes_per_call": lin_call_b,
+                       "hbm_gbs": lin_call_b / (avg["wgrad_fold"] * 1e-3) / 1e9},
+    }
+    traffic = load_traffic()
+    roofline = {"kernel": "fold_vec_kernel<bf16> (dominant: 8 launches per step)",
+                "bound": "hbm", "achieved": fold_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": fold_gbs / pk["hbm_gbs"], "peak_source": pk["source"],
+                "traffic": traffic.get("fold_bf16")}
+
+    # ---- end to end through the host-buffer entry points --------------------------------------
+    e2e = None
+    if rank == 0 or world > 1:
+        e2e = run_e2e(adama, dev, local, n, NA, NB, T, d_in, d_out, w, m, v, wB, mB, vB,
+                      max(1, min(args.steps, 3)), flat_b + lin_b, world, dist)
+
+    cpu_base = None
+    peak_mem = None
+    if rank == 0:
+        peak_mem = memory_report(adama, dev, local, T, d_in, d_out, Xs[0], dYs[0])
+        if world == 1 and not args.no_cpu_baseline:
+            cpu_base = time_oracle(1 << 25, 512, 512, 1024, 2, 1)
+            cpu_base = {k: cpu_base[k] for k in ("value", "unit", "cores", "kind", "sample",
+                                                 "seconds_per_sample_step")}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 (bf16 inputs on the fused path)",
+            "data": "synthetic",
+            "config": {"workload": f"headline: flat {n}-param buffer (bf16 grads, N={NA}) fold+apply, "
+                                   f"then linear {d_in}x{d_out} with {T} tokens (N={NB}) fused "
+                                   "wgrad+fold + apply",
+                       "l2": "inputs larger than L2, no flush", "replicas": world},
+            "fold_apply_GBps": (flat_b / ((sum(dur["fold"]) + sum(dur["apply"])) / args.steps * 1e-3)) / 1e9,
+            "wgrad_fold_TFLOPps": wgrad_tf,
+            "roofline": roofline, "roofline_kernels": roof_kernels,
+            "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks, "peak_memory": peak_mem,
+        }
+        print(json.dumps(line), flush=True)
+    optA.close()
+    optB.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def load_traffic():
+    """Per-launch DRAM traffic (bytes) from the committed ncu summary, keyed by kernel."""
+    p = ROOT / "profiles" / "traffic.json"
+    if p.exists():
+        try:
+            return json.loads(p.read_text())
+        except ValueError:
+            return {}
+    return {}
+
+
+def run_e2e(adama, dev, local, n, NA, NB, T, d_in, d_out, w, m, v, wB, mB, vB, steps, step_bytes,
+            world, dist):
+    """The same step through the host-buffer entry points: every gradient, X and dY comes from
+    pinned host memory and the updated weights are read back, all inside the timed region."""
+    optA = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=local)
+    optB = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=local)
+    g_host = [wl.normal((n,), wl.CONFIG2.grad_std, torch.bfloat16, 31 + i).pin_memory()
+              for i in range(2)]
+    X_host = wl.normal((T, d_in), 1.0, torch.bfloat16, 41).pin_memory()
+    dY_host = wl.normal((T, d_out), 1e-2, torch.bfloat16, 42).pin_memory()
+    w_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    wB_host = torch.empty(d_in * d_out, dtype=torch.float32).pin_memory()
+    staging = torch.empty(max(256 << 20, 2 * T * (d_in + d_out) + 512), dtype=torch.uint8,
+                          device=dev)
+
+    def step():
+        optA.begin_minibatch(NA)
+        for i in range(NA):
+            optA.fold_host(g_host[i & 1], m, v, staging)
+        optA.apply_to_host(w, m, v, wl.LR, w_host)
+        optB.begin_minibatch(NB)
+        for i in range(NB):
+            optB.linear_wgrad_fold_host(X_host, dY_host, mB, vB, staging)
+        optB.apply_to_host(wB, mB, vB, wl.LR, wB_host)
+
+    step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / steps
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    optA.sync_status()
+    optB.sync_status()
+    optA.close()
+    optB.close()
+    h2d = NA * n * 2 + NB * 2 * T * (d_in + d_out)
+    d2h = 4 * n + 4 * d_in * d_out
+    return {"value": world * step_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "steps": steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "api": "adama_fold_host / adama_linear_wgrad_fold_host / adama_apply_to_host"}
+
+
+def memory_report(adama, dev, local, T, d_in, d_out, X, dY):
+    """Peak device memory of one micro-batch of the linear layer with the fused kernel (no
+    gradient buffer) and with a materialised fp32 gradient folded by adama_fold."""
+    opt = adama.AdamA(device=local)
+    opt.begin_minibatch(1)
+    mB = torch.zeros(d_in, d_out, device=dev)
+    vB = torch.zeros(d_in, d_out, device=dev)
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats(dev)
+    base = torch.cuda.memory_allocated(dev)
+    opt.linear_wgrad_fold(X, dY, mB, vB)
+    torch.cuda.synchronize()
+    fused = torch.cuda.max_memory_allocated(dev) - base
+    torch.cuda.reset_peak_memory_stats(dev)
+    G = torch.empty(d_in, d_out, dtype=torch.float32, device=dev)  # the buffer AdamA's pipeline assigns
+    try:
+        torch.mm(X.t(), dY, out_dtype=torch.float32, out=G)
+    except (TypeError, RuntimeError):
+        G.zero_()  # the buffer is what is being measured, not its contents
+    opt.fold(G.view(-1), mB.view(-1), vB.view(-1))
+    torch.cuda.synchronize()
+    mat = torch.cuda.max_memory_allocated(dev) - base
+    del G
+    opt.close()
+    return {"layer": f"{d_in}x{d_out}", "extra_bytes_fused": int(fused),
+            "extra_bytes_materialised_gradient": int(mat),
+            "note": "bytes above the resident state and inputs during one micro-batch of the layer"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
