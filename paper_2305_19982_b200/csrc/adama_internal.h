@@ -22,8 +22,8 @@ struct ApplyConstants {
     float inv_bc2;   // 1 / (1 - beta2^t)
     float eps;       // eps
     float beta1_hi;  // beta1 = beta1_hi + beta1_lo to ~1e-15: the decay m*beta1 is
-    float beta1_lo;  // formed as fma(m, lo, m*hi), free of a per-step bias that
-    float beta2_hi;  // would otherwise build up over ~1/(1-beta) steps
+    float beta1_lo;  // formed as fma(m, hi, m*lo), free of the per-step bias of a
+    float beta2_hi;  // plain fp32 beta that would build up over ~1/(1-beta) steps
     float beta2_lo;
 };
 

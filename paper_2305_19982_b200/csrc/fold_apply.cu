@@ -126,8 +126,11 @@ fold_scalar_kernel(const G *__restrict__ grad, float *__restrict__ m, float *__r
 __device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
     float denom = sqrtf(v * c.inv_bc2) + c.eps;  // IEEE sqrt
     w = fmaf(-c.step, m / denom, w);             // IEEE division
-    m = fmaf(m, c.beta1_lo, m * c.beta1_hi);
-    v = fmaf(v, c.beta2_lo, v * c.beta2_hi);
+    // beta = hi + lo: the small product is rounded first (its error is ~1e-15 relative to
+    // the result), then one fma rounds x*hi + x*lo once.  The other order would round
+    // x*hi first and lose the sub-ulp correction every time.
+    m = fmaf(m, c.beta1_hi, m * c.beta1_lo);
+    v = fmaf(v, c.beta2_hi, v * c.beta2_lo);
 }
 
 template <int UNROLL>
