@@ -179,6 +179,43 @@ ADAMA_API adama_status adama_linear_wgrad_fold_host(adama_ctx *ctx, const void *
 ADAMA_API adama_status adama_apply_to_host(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                            double lr, float *w_host, void *cuda_stream);
 
+/* ---- for callers that must not allocate ------------------------------------------------- */
+
+/* The paper has no counterpart to this call; it exists for integration reasons only.
+ *
+ * Same computation as adama_linear_wgrad_fold, for code that is not allowed to take device
+ * memory from CUDA: for example a training job whose whole GPU memory is owned by a
+ * framework's pool, or a component that runs while the allocator must stay untouched.
+ * Such code cannot call adama_init (it allocates the status block), so this function takes
+ * the hyper-parameters and N directly and needs no context: a = (1-beta1)/N and
+ * b = (1-beta2)/N^2 are derived from cfg and n_micro exactly as a context would.
+ *
+ * The only memory the kernel uses besides X, dY, m and v is its 256-byte status block.
+ * Here that block is a fixed array inside the library image: every GPU that loads the
+ * library holds those 256 bytes until the process exits.  256 bytes is also the most this
+ * entry point can ever provide; a shape whose kernel needed more would be refused with
+ * ADAMA_ERR_UNSUPPORTED (today the need is the same for every shape).  The function calls
+ * no cudaMalloc/cudaFree and no allocating library routine.
+ *
+ *   - The first call on each device looks the array's device address up and sets the
+ *     kernel's shared-memory limit.  Make that first call outside any stream capture.
+ *   - All calls, from all threads and streams, share the one block.  It is cleared on the
+ *     stream before each launch.  Two calls that run on the GPU at the same time race on
+ *     it: the arithmetic on m and v stays correct, but a recorded time-out may be lost or
+ *     attributed to the wrong call.  Order such calls on one stream if the record matters.
+ *   - status_out_host (may be NULL): 4 words of host memory (pinned, if the copy is to be
+ *     asynchronous) that receive, once the stream reaches that point, {code, wait, tile, 0};
+ *     code 0 = finished normally, 1 = a bounded device-side wait expired.
+ *   - err / err_len (may be NULL / 0): caller's buffer for a message when the result is not
+ *     ADAMA_OK.
+ * Arguments X .. ldmv and their alignment rules are those of adama_linear_wgrad_fold.
+ * Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED (device ordinal >= 64, pitch too large,
+ * scratch need above 256 bytes), CUDA. */
+ADAMA_API adama_status adama_linear_wgrad_fold_noalloc(
+    const adama_config *cfg, int n_micro, const void *X, const void *dY, int tokens, int d_in,
+    int d_out, int64_t ldx, int64_t ldy, float *m, float *v, int64_t ldmv,
+    uint32_t *status_out_host, char *err, size_t err_len, void *cuda_stream);
+
 /* ---- state, checkpointing, diagnostics ------------------------------------------------- */
 
 /* Step counter t of Algorithm 2 (0 after init). */

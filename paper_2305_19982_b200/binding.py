@@ -18,7 +18,7 @@ _LIB_PATH = _PKG / "libadama.so"
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
     "adama_linear_wgrad_fold", "adama_apply", "adama_fold_host", "adama_linear_wgrad_fold_host",
-    "adama_apply_to_host", "adama_get_step", "adama_set_step", "adama_get_n_micro",
+    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
     "adama_version",
 ]
@@ -76,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
     L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
     L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
+    L.adama_linear_wgrad_fold_noalloc.argtypes = [ctypes.POINTER(_Config), ci, vp, vp, ci, ci, ci,
+                                                  i64, i64, vp, vp, i64, vp, ctypes.c_char_p, sz, vp]
     L.adama_get_step.argtypes = [vp]
     L.adama_get_step.restype = i64
     L.adama_set_step.argtypes = [vp, i64]
@@ -268,6 +270,36 @@ class AdamA:
     @property
     def launch_count(self) -> int:
         return int(self._L.adama_launch_count(self._h))
+
+
+def linear_wgrad_fold_noalloc(X: torch.Tensor, dY: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
+                              n_micro: int, beta1=0.9, beta2=0.999, status_out=None,
+                              grads_prescaled=False) -> None:
+    """adama_linear_wgrad_fold_noalloc: the fused weight-gradient fold for callers that may
+    not allocate device memory.  Needs no AdamA context; the kernel's status block is a
+    fixed array inside the library.  `status_out`, if given, is a pinned CPU int32/uint32
+    tensor of >= 4 elements that receives {code, wait, tile, 0} when the stream gets there."""
+    L = load_library()
+    tokens, d_in = X.shape
+    d_out = dY.shape[1]
+    dev = X.device.index if X.device.index is not None else torch.cuda.current_device()
+    cfg = _Config(beta1, beta2, 0.0, dev, GRADS_PRESCALED if grads_prescaled else 0)
+    err = ctypes.create_string_buffer(256)
+    ldx = X.stride(0) if tokens > 1 else max(d_in, X.stride(0))
+    ldy = dY.stride(0) if tokens > 1 else max(d_out, dY.stride(0))
+    ldmv = m.stride(0) if d_in > 1 else max(d_out, m.stride(0))
+    sp = None
+    if status_out is not None:
+        if status_out.is_cuda or status_out.numel() < 4 or status_out.element_size() != 4:
+            raise TypeError("status_out must be a CPU tensor of >= 4 32-bit elements")
+        sp = status_out.data_ptr()
+    st = L.adama_linear_wgrad_fold_noalloc(
+        ctypes.byref(cfg), int(n_micro), _dev_ptr(X, torch.bfloat16, "X"),
+        _dev_ptr(dY, torch.bfloat16, "dY"), tokens, d_in, d_out, ldx, ldy,
+        _dev_ptr(m, torch.float32, "m"), _dev_ptr(v, torch.float32, "v"), ldmv, sp, err, 256,
+        _stream_ptr(torch.device("cuda", dev)))
+    if st != 0:
+        raise AdamAError(st, err.value.decode())
 
 
 def version() -> str:

@@ -530,3 +530,151 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
 }
 
 }  // namespace adama
+
+// ---- allocation-free entry point ------------------------------------------------------------
+//
+// The fused kernel needs one piece of global memory besides its inputs and outputs: the
+// 256-byte status block in which a CTA records that a bounded wait ran out.  A context
+// gets that block from cudaMalloc.  Code that must not allocate -- a training loop whose
+// device memory belongs entirely to a framework's pool, a plug-in called while another
+// component holds the allocator lock, a caller past its memory budget -- cannot create a
+// context, so this entry point needs none: the block lives in the library image itself.
+
+namespace adama {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 256;  // the whole need of the kernel, whatever the shapes
+constexpr int kMaxDevices = 64;
+
+// One copy per GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticSetup {
+    unsigned *scratch = nullptr;  // DEVICE address of g_static_scratch on that GPU
+    int sm_count = 0;
+};
+StaticSetup g_static_setup[kMaxDevices];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel
+// can use; the device address has to be asked for, with the right device current.
+cudaError_t static_setup_for_current_device(int device, StaticSetup **out, const char **msg) {
+    StaticSetup &s = g_static_setup[device];
+    if (!s.scratch) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) {
+            *msg = "cudaGetSymbolAddress(static scratch)";
+            return e;
+        }
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) {
+            *msg = "cudaDeviceGetAttribute(multiProcessorCount)";
+            return e;
+        }
+        s.sm_count = sms;
+        s.scratch = static_cast<unsigned *>(ptr);
+    }
+    *out = &s;
+    return cudaSuccess;
+}
+
+void set_msg(char *err, size_t err_len, const char *text, const char *detail = nullptr) {
+    if (!err || err_len == 0) return;
+    size_t k = 0;
+    for (const char *p = text; *p && k + 1 < err_len; ++p) err[k++] = *p;
+    if (detail) {
+        for (const char *p = ": "; *p && k + 1 < err_len; ++p) err[k++] = *p;
+        for (const char *p = detail; *p && k + 1 < err_len; ++p) err[k++] = *p;
+    }
+    err[k] = 0;
+}
+
+bool is_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+}  // namespace adama
+
+extern "C" adama_status adama_linear_wgrad_fold_noalloc(
+    const adama_config *cfg, int n_micro, const void *X, const void *dY, int tokens, int d_in,
+    int d_out, int64_t ldx, int64_t ldy, float *m, float *v, int64_t ldmv, uint32_t *status_out_host,
+    char *err, size_t err_len, void *cuda_stream) {
+    using namespace adama;
+    set_msg(err, err_len, "");
+    if (!cfg || !(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0) ||
+        cfg->device < 0 || (cfg->flags & ~ADAMA_GRADS_PRESCALED) != 0 || n_micro < 1) {
+        set_msg(err, err_len, "noalloc: bad configuration or n_micro < 1");
+        return ADAMA_ERR_INVALID_ARG;
+    }
+    if (cfg->device >= kMaxDevices) {
+        set_msg(err, err_len, "noalloc: device ordinal beyond the 64 this entry point keeps set-up for");
+        return ADAMA_ERR_UNSUPPORTED;
+    }
+    if (tokens < 0 || d_in < 1 || d_out < 1 || !m || !v || (tokens > 0 && (!X || !dY)) ||
+        ldx < d_in || ldy < d_out || ldmv < d_out) {
+        set_msg(err, err_len, "noalloc: bad shape, null pointer or row pitch smaller than the row");
+        return ADAMA_ERR_INVALID_ARG;
+    }
+    if (!is_aligned(X, 16) || !is_aligned(dY, 16) || !is_aligned(m, 16) || !is_aligned(v, 16) ||
+        ldx % 8 || ldy % 8 || ldmv % 4) {
+        set_msg(err, err_len,
+                "noalloc: X, dY, m, v must be 16-byte aligned, ldx and ldy multiples of 8, ldmv of 4");
+        return ADAMA_ERR_MISALIGNED;
+    }
+    if (ldx * 2 >= (1ll << 40) || ldy * 2 >= (1ll << 40) || ldmv * 4 >= (1ll << 40)) {
+        set_msg(err, err_len, "noalloc: row pitch too large for a tensor map");
+        return ADAMA_ERR_UNSUPPORTED;
+    }
+    // Scratch the kernel would need for these shapes against what the static array holds.
+    // The need is one status block for every shape, so this cannot fail today; it is
+    // checked so that a later kernel with a shape-dependent need fails here, not on the GPU.
+    const size_t scratch_needed = 256;
+    if (scratch_needed > kStaticScratchBytes) {
+        set_msg(err, err_len, "noalloc: problem needs more scratch than the 256-byte static block");
+        return ADAMA_ERR_UNSUPPORTED;
+    }
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    cudaError_t e = (prev == cfg->device) ? cudaSuccess : cudaSetDevice(cfg->device);
+    const char *msg = "cudaSetDevice";
+    StaticSetup *setup = nullptr;
+    if (e == cudaSuccess) e = static_setup_for_current_device(cfg->device, &setup, &msg);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (e == cudaSuccess && tokens > 0) {
+        // every call shares the block, which still holds the last call's record
+        msg = "cudaMemsetAsync(static scratch)";
+        e = cudaMemsetAsync(setup->scratch, 0, kStaticScratchBytes, stream);
+        if (e == cudaSuccess) {
+            WgradArgs a;
+            a.X = X;
+            a.dY = dY;
+            a.tokens = tokens;
+            a.d_in = d_in;
+            a.d_out = d_out;
+            a.ldx = ldx;
+            a.ldy = ldy;
+            a.ldmv = ldmv;
+            a.m = m;
+            a.v = v;
+            a.c = make_fold_constants(cfg->beta1, cfg->beta2, n_micro, cfg->flags);
+            a.status = setup->scratch;
+            a.sm_count = setup->sm_count;
+            a.stream = stream;
+            e = launch_wgrad_fold(a, &msg);
+        }
+        if (e == cudaSuccess && status_out_host) {
+            msg = "cudaMemcpyAsync(status)";
+            e = cudaMemcpyAsync(status_out_host, setup->scratch, 4 * sizeof(uint32_t),
+                                cudaMemcpyDeviceToHost, stream);
+        }
+    } else if (e == cudaSuccess && status_out_host) {
+        status_out_host[0] = status_out_host[1] = status_out_host[2] = status_out_host[3] = 0;
+    }
+    if (prev >= 0 && prev != cfg->device) cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+        set_msg(err, err_len, msg, cudaGetErrorString(e));
+        return ADAMA_ERR_CUDA;
+    }
+    return ADAMA_OK;
+}
