@@ -319,10 +319,12 @@ def run_ours(args):
                        "unit": "TFLOP/s", "frac": wgrad_tf / pk["bf16_tflops"],
                        "frac_of_sustained": wgrad_tf / pk["bf16_tflops_sustained"],
                        "ms": avg["wgrad_fold"], "flops_per_call": 2.0 * T * d_in * d_out,
-                       "hbm_bytes_per_call": lin_call_b,
+                       "hbm_bytes_per_call": lin_call_b, "traffic": None,
                        "hbm_gbs": lin_call_b / (avg["wgrad_fold"] * 1e-3) / 1e9},
     }
     traffic = load_traffic()
+    for key in roof_kernels:
+        roof_kernels[key]["traffic"] = traffic.get(key)
     roofline = {"kernel": "fold_vec_kernel<bf16> (dominant: 8 launches per step)",
                 "bound": "hbm", "achieved": fold_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": fold_gbs / pk["hbm_gbs"], "peak_source": pk["source"],
@@ -330,7 +332,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry points --------------------------------------
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.no_e2e:
         e2e = run_e2e(adama, dev, local, n, NA, NB, T, d_in, d_out, w, m, v, wB, mB, vB,
                       max(1, min(args.steps, 3)), flat_b + lin_b, world, dist)
 
@@ -367,14 +369,24 @@ def run_ours(args):
 
 
 def load_traffic():
-    """Per-launch DRAM traffic (bytes) from the committed ncu summary, keyed by kernel."""
+    """Per-launch DRAM traffic (bytes) from the committed ncu summaries, keyed by kernel; an
+    entry counts only while the kernel's source file is the one the counters were taken on."""
+    import hashlib
     p = ROOT / "profiles" / "traffic.json"
-    if p.exists():
-        try:
-            return json.loads(p.read_text())
-        except ValueError:
-            return {}
-    return {}
+    out = {}
+    if not p.exists():
+        return out
+    try:
+        data = json.loads(p.read_text())
+    except ValueError:
+        return out
+    for key, ent in data.items():
+        if not isinstance(ent, dict):
+            continue
+        src = ROOT / ent.get("source", "")
+        if src.is_file() and hashlib.sha256(src.read_bytes()).hexdigest() == ent.get("sha256"):
+            out[key] = ent.get("bytes_per_launch")
+    return out
 
 
 def run_e2e(adama, dev, local, n, NA, NB, T, d_in, d_out, w, m, v, wB, mB, vB, steps, step_bytes,
@@ -466,6 +478,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
