@@ -8,39 +8,48 @@
 // the TMA unit as reduce-add stores, so m and v are read-modified-written at the
 // L2 and the SM never waits on a global load.
 //
-// Persistent kernel, one CTA per SM, 192 threads:
-//   warp 0      TMA producer: X and dY tiles -> 4-stage shared-memory ring
-//   warp 1      MMA issuer (single thread) + owner of the 512 TMEM columns
-//   warps 2..5  epilogue, one TMEM lane quarter each
-// The 512 TMEM columns hold two 128x256 fp32 accumulators, so the epilogue of tile
-// i overlaps the main loop of tile i+1.
+// Persistent kernel, 192 threads per CTA, CTAs working in pairs (a cluster of two on
+// the two SMs of a TPC, tcgen05 cta_group::2): a pair owns a 256x256 output tile,
+// each CTA its 128 rows.  Per 64-token stage a CTA loads its own 128 rows of X^T and
+// only HALF of the dY tile (128 of the 256 columns); the tensor cores of both SMs
+// read both halves.  That is 64 bytes of operands per tensor-core clock and SM
+// instead of 96 for a lone 128x256 tile, and leaves room for a 6-stage ring.
+//   warp 0      TMA producer: operand tiles -> shared-memory ring (both CTAs)
+//   warp 1      MMA issuer (one thread of the pair's first CTA) + TMEM allocation
+//   warps 2..5  epilogue, one TMEM lane quarter each (both CTAs)
+// The 512 TMEM columns hold two 128x256 fp32 accumulators per CTA, so the epilogue of
+// tile i overlaps the main loop of tile i+1.  (A one-CTA variant, 128x256 tiles and a
+// 4-stage ring, is kept as a template instance for comparison.)
 //
 // Operand layout.  The contraction runs over tokens, the strided dimension of both
 // row-major inputs, so both operands are "MN-major": a TMA box of 64 features x 64
 // tokens lands as 64 rows of 128 bytes (one token per row) under the 128-byte
-// swizzle; a 128-row A tile is two such boxes, a 256-column B tile four.  The
-// shared-memory matrix descriptor states: 8-token groups 1024 bytes apart (stride
-// byte offset), 64-feature groups one box (8192 bytes) apart (leading byte offset).
+// swizzle.  The shared-memory matrix descriptor states: 8-token groups 1024 bytes
+// apart (stride byte offset), 64-feature groups one box (8192 bytes) apart (leading
+// byte offset).
+//
+// Synchronisation of a pair: the first CTA's "full" barrier of a stage counts the
+// bytes of both CTAs' loads; when the MMAs that read a stage retire, tcgen05.commit
+// arrives on the "empty" barrier of each CTA; the same for accumulator-full; the
+// eight epilogue warps of the pair arrive on the first CTA's accumulator-empty
+// barrier.  No load uses cluster multicast.
 //
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the kernel
 // records a code in the status block, all roles drain and leave, TMEM is freed.
 #include <cuda.h>
+
+#include <cstdlib>
 
 #include "adama_internal.h"
 
 namespace adama {
 namespace {
 
-constexpr int BM = 128;     // tile rows    (d_in  direction) = UMMA M
 constexpr int BN = 256;     // tile columns (d_out direction) = UMMA N
 constexpr int BK = 64;      // tokens per pipeline stage
 constexpr int UMMA_K = 16;  // tokens per tcgen05.mma (bf16)
-constexpr int STAGES = 4;
-constexpr int GROUP = 64;                                // features per 128-byte swizzled row
-constexpr int BOX_BYTES = GROUP * BK * 2;                // 8192
-constexpr int A_STAGE_BYTES = (BM / GROUP) * BOX_BYTES;  // 16384
-constexpr int B_STAGE_BYTES = (BN / GROUP) * BOX_BYTES;  // 32768
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int GROUP = 64;   // features per 128-byte swizzled row
+constexpr int BOX_BYTES = GROUP * BK * 2;               // 8192
 constexpr int EPI_COLS = 32;                            // fp32 columns per reduce box (128 B)
 constexpr int EPI_ROWS = 32;                            // one TMEM lane quarter
 constexpr int EPI_BUF_BYTES = EPI_ROWS * EPI_COLS * 4;  // 4096
@@ -49,25 +58,39 @@ constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
 constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
-
-constexpr int SMEM_RING_OFF = 0;
-constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
-constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
+constexpr int MAX_STAGES = 6;
 constexpr int SMEM_BAR_BYTES = 256;
-constexpr int SMEM_BYTES = SMEM_BAR_OFF + SMEM_BAR_BYTES + 1024;  // + slack for 1024-B alignment
-static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+// Per-variant geometry: CTAS = CTAs cooperating on one tile (1 or 2).
+template <int CTAS>
+struct Geo {
+    static constexpr int ROWS_PER_CTA = 128;                 // TMEM lanes
+    static constexpr int TILE_M = ROWS_PER_CTA * CTAS;       // UMMA M
+    static constexpr int B_COLS_PER_CTA = BN / CTAS;         // dY columns this CTA stages
+    static constexpr int A_BOXES = ROWS_PER_CTA / GROUP;     // 2
+    static constexpr int B_BOXES = B_COLS_PER_CTA / GROUP;   // 4 or 2
+    static constexpr int A_STAGE_BYTES = A_BOXES * BOX_BYTES;
+    static constexpr int B_STAGE_BYTES = B_BOXES * BOX_BYTES;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KB or 32 KB
+    static constexpr int STAGES = CTAS == 1 ? 4 : 6;
+    static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
+    static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
+    static constexpr int SMEM_BYTES = SMEM_BAR_OFF + SMEM_BAR_BYTES + 1024;  // + alignment slack
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(STAGES <= MAX_STAGES, "barrier block");
+    // tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both
+    // MN-major, N = 256, M = 128 per participating CTA.
+    static constexpr uint32_t INSTR_DESC = (1u << 4)     // D format: f32
+                                           | (1u << 7)   // A format: bf16
+                                           | (1u << 10)  // B format: bf16
+                                           | (1u << 15)  // A is MN-major
+                                           | (1u << 16)  // B is MN-major
+                                           | ((uint32_t)(BN >> 3) << 17) |
+                                           ((uint32_t)(TILE_M >> 4) << 24);
+};
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr unsigned long long kDrainLimitNs = 20000000ull;   // 20 ms
-
-// tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both
-// MN-major, N = 256, M = 128.
-constexpr uint32_t kInstrDesc = (1u << 4)      // D format: f32
-                                | (1u << 7)    // A format: bf16
-                                | (1u << 10)   // B format: bf16
-                                | (1u << 15)   // A is MN-major
-                                | (1u << 16)   // B is MN-major
-                                | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 // ---- PTX wrappers --------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -78,11 +101,31 @@ __device__ __forceinline__ unsigned long long globaltimer() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `addr` (a shared::cta address) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;"
+                 ::: "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// arrive on a barrier given by its shared::cluster address (own CTA or the partner)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
+                 : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
@@ -112,13 +155,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
+// TMA tile load into this CTA's shared memory; `bar` is a shared::cluster address and,
+// for CTAS == 2, may name the partner CTA's barrier.
+template <int CTAS>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
                                             uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+            "l"(map), "r"(x), "r"(y), "r"(bar)
+            : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+            "l"(map), "r"(x), "r"(y), "r"(bar)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int x, int y,
                                                   uint32_t src) {
@@ -147,19 +201,62 @@ __device__ __forceinline__ void tc_fence_before() {
 __device__ __forceinline__ void tc_fence_after() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                     bar)
-                 : "memory");
+// Arrive on `cluster_bar` (shared::cluster address) once all MMAs issued so far by this
+// thread have retired.
+template <int CTAS>
+__device__ __forceinline__ void tc_commit(uint32_t cluster_bar) {
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                         cluster_bar)
+                     : "memory");
+    } else {
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                         cluster_bar)
+                     : "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b,
                                        uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+            "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+            "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+template <int CTAS>
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem) {
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                     "n"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                     "n"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+}
+template <int CTAS>
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr) {
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "n"(TMEM_COLS)
+                     : "memory");
+    } else {
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "n"(TMEM_COLS)
+                     : "memory");
+    }
 }
 // 32 lanes x 32 consecutive fp32 columns: thread i receives TMEM lane (base lane + i).
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -195,8 +292,8 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
 }
 
 struct Barriers {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
     uint64_t acc_full[ACC_STAGES];
     uint64_t acc_empty[ACC_STAGES];
     uint64_t drain;
@@ -214,22 +311,28 @@ __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars,
     }
 }
 
+template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   const __grid_constant__ CUtensorMap map_dy,
                   const __grid_constant__ CUtensorMap map_m,
                   const __grid_constant__ CUtensorMap map_v, int tokens, int d_in, int d_out,
                   float a, float b, unsigned *status) {
+    using G = Geo<CTAS>;
+    constexpr int STAGES = G::STAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;  // swizzled tiles need 1024-B alignment
     uint8_t *smem = smem_raw + (base - raw_addr);
-    Barriers *bars = reinterpret_cast<Barriers *>(smem + SMEM_BAR_OFF);
+    Barriers *bars = reinterpret_cast<Barriers *>(smem + G::SMEM_BAR_OFF);
     volatile int *abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int tiles_m = (d_in + BM - 1) / BM;
+    const uint32_t rank = (CTAS == 1) ? 0u : cluster_ctarank();  // position in the pair
+    const int group = blockIdx.x / CTAS;                           // which pair
+    const int num_groups = gridDim.x / CTAS;
+    const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
     const int tiles_n = (d_out + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_n;
     const int num_kb = (tokens + BK - 1) / BK;
@@ -241,35 +344,30 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         }
         for (int s = 0; s < ACC_STAGES; ++s) {
             mbar_init(smem_u32(&bars->acc_full[s]), 1);
-            mbar_init(smem_u32(&bars->acc_empty[s]), EPI_WARPS);
+            mbar_init(smem_u32(&bars->acc_empty[s]), EPI_WARPS * CTAS);
         }
         mbar_init(smem_u32(&bars->drain), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         smem_u32(&bars->tmem_base)),
-                     "n"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc<CTAS>(smem_u32(&bars->tmem_base));
     tc_fence_before();
     __syncthreads();
+    if constexpr (CTAS == 2) cluster_sync_all();  // the partner's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (every CTA) ----------------
         int stage = 0;
         uint32_t phase = 0;
         uint32_t armed = 0;        // bit s: stage s has been armed at least once
         uint32_t last_parity = 0;  // bit s: parity of the phase last armed on stage s
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int m0 = (tile % tiles_m) * BM;
-            const int n0 = (tile / tiles_m) * BN;
+        for (int tile = group; tile < num_tiles && ok; tile += num_groups) {
+            const int m0 = (tile % tiles_m) * G::TILE_M + (int)rank * G::ROWS_PER_CTA;
+            const int n0 = (tile / tiles_m) * BN + (int)rank * G::B_COLS_PER_CTA;
             for (int kb = 0; kb < num_kb; ++kb) {
                 ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
@@ -278,17 +376,19 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     break;
                 }
                 if (lane == 0) {
-                    const uint32_t bar = smem_u32(&bars->full[stage]);
-                    const uint32_t sa = base + SMEM_RING_OFF + stage * STAGE_BYTES;
-                    const uint32_t sb = sa + A_STAGE_BYTES;
+                    const uint32_t own_bar = smem_u32(&bars->full[stage]);
+                    // the pair's loads are counted by the first CTA's barrier
+                    const uint32_t bar = (CTAS == 1) ? own_bar : map_to_cta(own_bar, 0);
+                    const uint32_t sa = base + stage * G::STAGE_BYTES;
+                    const uint32_t sb = sa + G::A_STAGE_BYTES;
                     // out-of-range parts of a box are zero-filled and still counted
-                    mbar_arrive_expect_tx(bar, STAGE_BYTES);
+                    if (rank == 0) mbar_arrive_expect_tx(own_bar, G::STAGE_BYTES * CTAS);
 #pragma unroll
-                    for (int j = 0; j < BM / GROUP; ++j)
-                        tma_load_2d(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK, bar);
+                    for (int j = 0; j < G::A_BOXES; ++j)
+                        tma_load_2d<CTAS>(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK, bar);
 #pragma unroll
-                    for (int j = 0; j < BN / GROUP; ++j)
-                        tma_load_2d(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK, bar);
+                    for (int j = 0; j < G::B_BOXES; ++j)
+                        tma_load_2d<CTAS>(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK, bar);
                 }
                 armed |= 1u << stage;
                 last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
@@ -299,7 +399,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 }
             }
         }
-        if (*abort_flag) {
+        if (*abort_flag && rank == 0) {
             // leave no copy in flight behind: wait (bounded) for every armed stage to land
             int never = 0;
             for (int s = 0; s < STAGES; ++s)
@@ -308,72 +408,83 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                               kDrainLimitNs);
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        int it = 0;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-            const int as = it & 1;
-            const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-            ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) {
-                if (lane == 0) record_timeout(status, bars, 2, (unsigned)tile);
-                break;
-            }
-            tc_fence_after();
-            const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
-            for (int kb = 0; kb < num_kb; ++kb) {
-                ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag);
+        // ---------------- MMA issuer (first CTA of the pair only) ----------------
+        if (rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = group; tile < num_tiles && ok; tile += num_groups, ++it) {
+                const int as = it & 1;
+                const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+                ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) {
-                    if (lane == 0) record_timeout(status, bars, 3, (unsigned)tile);
+                    if (lane == 0) record_timeout(status, bars, 2, (unsigned)tile);
                     break;
                 }
                 tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t sa = base + SMEM_RING_OFF + stage * STAGE_BYTES;
-                    const uint32_t sb = sa + A_STAGE_BYTES;
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // 16 tokens further = 16 rows of 128 bytes
-                        const uint64_t da = make_smem_desc(sa + k * (UMMA_K * 128));
-                        const uint64_t db = make_smem_desc(sb + k * (UMMA_K * 128));
-                        tc_mma(tmem_d, da, db, kInstrDesc, (kb | k) != 0 ? 1u : 0u);
+                const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) {
+                        if (lane == 0) record_timeout(status, bars, 3, (unsigned)tile);
+                        break;
                     }
-                    tc_commit(smem_u32(&bars->empty[stage]));  // stage free once these MMAs retire
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t sa = base + stage * G::STAGE_BYTES;
+                        const uint32_t sb = sa + G::A_STAGE_BYTES;
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            // 16 tokens further = 16 rows of 128 bytes
+                            const uint64_t da = make_smem_desc(sa + k * (UMMA_K * 128));
+                            const uint64_t db = make_smem_desc(sb + k * (UMMA_K * 128));
+                            tc_mma<CTAS>(tmem_d, da, db, G::INSTR_DESC, (kb | k) != 0 ? 1u : 0u);
+                        }
+                        // the stage is free, in every CTA of the pair, once these MMAs retire
+                        const uint32_t e = smem_u32(&bars->empty[stage]);
+#pragma unroll
+                        for (int r = 0; r < CTAS; ++r)
+                            tc_commit<CTAS>(CTAS == 1 ? e : map_to_cta(e, r));
+                    }
+                    __syncwarp();
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                }
+                if (ok && lane == 0) {
+                    const uint32_t f = smem_u32(&bars->acc_full[as]);
+#pragma unroll
+                    for (int r = 0; r < CTAS; ++r) tc_commit<CTAS>(CTAS == 1 ? f : map_to_cta(f, r));
                 }
                 __syncwarp();
-                if (++stage == STAGES) {
-                    stage = 0;
-                    phase ^= 1;
-                }
             }
-            if (ok && lane == 0) tc_commit(smem_u32(&bars->acc_full[as]));
-            __syncwarp();
-        }
-        if (*abort_flag) {
-            // let issued MMAs retire before TMEM is given back
-            if (lane == 0) tc_commit(smem_u32(&bars->drain));
-            __syncwarp();
-            int never = 0;
-            mbar_wait(smem_u32(&bars->drain), 0, &never, kDrainLimitNs);
+            if (*abort_flag) {
+                // let issued MMAs retire before TMEM is given back
+                if (lane == 0) tc_commit<CTAS>(smem_u32(&bars->drain));
+                __syncwarp();
+                int never = 0;
+                mbar_wait(smem_u32(&bars->drain), 0, &never, kDrainLimitNs);
+            }
         }
     } else {
         // ---------------- epilogue: TMEM -> a*G, b*G^2 -> TMA reduce-add into m, v ----------
         const int q = warp & 3;  // TMEM lane quarter this warp may read
-        const uint32_t sm_m = base + SMEM_EPI_OFF + (uint32_t)q * 2 * EPI_BUF_BYTES;
+        const uint32_t sm_m = base + G::SMEM_EPI_OFF + (uint32_t)q * 2 * EPI_BUF_BYTES;
         const uint32_t sm_v = sm_m + EPI_BUF_BYTES;
         // 128-byte swizzle: 16-byte chunk j of row r sits at chunk (j ^ (r & 7))
         const uint32_t row_off = (uint32_t)lane * 128u;
         const uint32_t sw = (uint32_t)(lane & 7);
         bool ok = true;
         int it = 0;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        for (int tile = group; tile < num_tiles && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-            const int row0 = (tile % tiles_m) * BM + q * EPI_ROWS;
+            const int row0 =
+                (tile % tiles_m) * G::TILE_M + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
             const int n0 = (tile / tiles_m) * BN;
             ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
@@ -429,10 +540,14 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     }
                 }
             }
-            // accumulator stage may now be overwritten by the MMA warp
+            // accumulator stage may now be overwritten by the pair's MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[as]));
+            if (lane == 0) {
+                const uint32_t e = smem_u32(&bars->acc_empty[as]);
+                if constexpr (CTAS == 1) mbar_arrive(e);
+                else mbar_arrive_cluster(map_to_cta(e, 0));
+            }
         }
         if (lane == 0) bulk_wait_all();  // reduce-adds complete before the CTA retires
         __syncwarp();
@@ -440,11 +555,12 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
 
     tc_fence_before();
     __syncthreads();
+    // neither CTA of a pair may retire while the other can still read its shared memory
+    // or signal its barriers
+    if constexpr (CTAS == 2) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                     "n"(TMEM_COLS)
-                     : "memory");
+        tmem_dealloc<CTAS>(tmem_base);
     }
 }
 
@@ -456,6 +572,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 bool g_attr_set = false;
+int g_variant = 0;  // 0 = not chosen yet, 1 = one-CTA tiles, 2 = CTA pairs
 
 // 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
 bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void *ptr,
@@ -489,6 +606,11 @@ cudaError_t wgrad_fold_setup(const char **msg) {
         }
         g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
+    if (!g_variant) {
+        // ADAMA_WGRAD_CTAS=1 selects the one-CTA tiling (for comparisons); default: pairs
+        const char *env = getenv("ADAMA_WGRAD_CTAS");
+        g_variant = (env && env[0] == '1') ? 1 : 2;
+    }
     return cudaSuccess;
 }
 
@@ -496,8 +618,11 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cudaError_t e = wgrad_fold_setup(msg);
     if (e != cudaSuccess) return e;
     if (!g_attr_set) {
-        e = cudaFuncSetAttribute(wgrad_fold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 SMEM_BYTES);
+        e = cudaFuncSetAttribute(wgrad_fold_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Geo<1>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(wgrad_fold_kernel<2>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::SMEM_BYTES);
         if (e != cudaSuccess) {
             *msg = "cudaFuncSetAttribute(wgrad_fold_kernel)";
             return e;
@@ -521,12 +646,32 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
         *msg = "cuTensorMapEncodeTiled rejected a tensor";
         return cudaErrorInvalidValue;
     }
-    const int tiles = ((p.d_in + BM - 1) / BM) * ((p.d_out + BN - 1) / BN);
-    const int grid = tiles < p.sm_count ? tiles : p.sm_count;
-    wgrad_fold_kernel<<<grid, NUM_THREADS, SMEM_BYTES, p.stream>>>(
-        map_x, map_dy, map_m, map_v, p.tokens, p.d_in, p.d_out, p.c.a, p.c.b, p.status);
+    const int tiles_n = (p.d_out + BN - 1) / BN;
     *msg = "wgrad_fold launch";
-    return cudaGetLastError();
+    if (g_variant == 1) {
+        const int tiles = ((p.d_in + Geo<1>::TILE_M - 1) / Geo<1>::TILE_M) * tiles_n;
+        const int grid = tiles < p.sm_count ? tiles : p.sm_count;
+        wgrad_fold_kernel<1><<<grid, NUM_THREADS, Geo<1>::SMEM_BYTES, p.stream>>>(
+            map_x, map_dy, map_m, map_v, p.tokens, p.d_in, p.d_out, p.c.a, p.c.b, p.status);
+        return cudaGetLastError();
+    }
+    const int tiles = ((p.d_in + Geo<2>::TILE_M - 1) / Geo<2>::TILE_M) * tiles_n;
+    const int pairs = p.sm_count / 2;
+    const int groups = tiles < pairs ? tiles : pairs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = Geo<2>::SMEM_BYTES;
+    cfg.stream = p.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_m, map_v, p.tokens,
+                              p.d_in, p.d_out, p.c.a, p.c.b, p.status);
 }
 
 }  // namespace adama
