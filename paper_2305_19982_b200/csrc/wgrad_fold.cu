@@ -79,14 +79,14 @@ struct Geo {
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(STAGES <= MAX_STAGES, "barrier block");
     // tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both
-    // MN-major, N = 256, M = 128 per participating CTA.
-    static constexpr uint32_t INSTR_DESC = (1u << 4)     // D format: f32
-                                           | (1u << 7)   // A format: bf16
-                                           | (1u << 10)  // B format: bf16
-                                           | (1u << 15)  // A is MN-major
-                                           | (1u << 16)  // B is MN-major
-                                           | ((uint32_t)(BN >> 3) << 17) |
-                                           ((uint32_t)(TILE_M >> 4) << 24);
+    // MN-major, M = 128 per participating CTA; N (bits 17..22, in units of 8) is added
+    // per work item.
+    static constexpr uint32_t INSTR_DESC_NO_N = (1u << 4)     // D format: f32
+                                                | (1u << 7)   // A format: bf16
+                                                | (1u << 10)  // B format: bf16
+                                                | (1u << 15)  // A is MN-major
+                                                | (1u << 16)  // B is MN-major
+                                                | ((uint32_t)(TILE_M >> 4) << 24);
 };
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
@@ -282,13 +282,19 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, float x, float y, fl
 }
 
 // Shared-memory matrix descriptor for an MN-major bf16 operand under the 128-byte
-// swizzle: start address, leading byte offset (between 64-feature groups), stride
-// byte offset (between 8-token groups), descriptor version 1, layout SWIZZLE_128B.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
-    constexpr uint64_t lbo = BOX_BYTES >> 4;  // 8192 B
-    constexpr uint64_t sbo = 1024 >> 4;       // 8 tokens x 128 B
-    return (uint64_t)((addr & 0x3ffff) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) |
-           (2ull << 61);
+// swizzle.  Low word: start address >> 4 (bits 0..13) and leading byte offset >> 4
+// (bits 16..29, the distance between 64-feature groups = one 8192-byte box).  High
+// word: stride byte offset >> 4 (bits 32..45, the distance between 8-token groups =
+// 1024 bytes), descriptor version 1 (bits 46..47), layout SWIZZLE_128B = 2 (bits 61..63).
+// Only the start address changes between MMAs, so the issuing thread keeps the low word
+// in a register and adds byte offsets >> 4 to it (no carry into bit 14: shared memory
+// is smaller than 256 KB).
+constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) {
+    return ((addr & 0x3ffffu) >> 4) | ((uint32_t)(BOX_BYTES >> 4) << 16);
+}
+__device__ __forceinline__ uint64_t smem_desc(uint32_t lo) {
+    return ((uint64_t)kDescHi << 32) | (uint64_t)lo;
 }
 
 struct Barriers {
@@ -311,13 +317,33 @@ __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars,
     }
 }
 
+// Work list of a launch.  Items [0, split_from) are full tiles (TILE_M x 256), numbered
+// with the row-tile index fastest.  Items from split_from on are the two 128-column halves
+// of the remaining full tiles: when the last round would occupy at most half of the CTA
+// groups, halving its tiles halves its duration (the token sum of each half is still
+// complete, so the square stays exact).
+struct WorkItem {
+    int m0, n0, width;
+};
+template <int CTAS>
+__device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m) {
+    int full = w, half = 0, width = BN;
+    if (w >= split_from) {
+        const int j = w - split_from;
+        full = split_from + (j >> 1);
+        half = j & 1;
+        width = BN / 2;
+    }
+    return {(full % tiles_m) * Geo<CTAS>::TILE_M, (full / tiles_m) * BN + half * (BN / 2), width};
+}
+
 template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   const __grid_constant__ CUtensorMap map_dy,
                   const __grid_constant__ CUtensorMap map_m,
                   const __grid_constant__ CUtensorMap map_v, int tokens, int d_in, int d_out,
-                  float a, float b, unsigned *status) {
+                  int split_from, int num_items, float a, float b, unsigned *status) {
     using G = Geo<CTAS>;
     constexpr int STAGES = G::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -333,8 +359,6 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     const int group = blockIdx.x / CTAS;                           // which pair
     const int num_groups = gridDim.x / CTAS;
     const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
-    const int tiles_n = (d_out + BN - 1) / BN;
-    const int num_tiles = tiles_m * tiles_n;
     const int num_kb = (tokens + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
@@ -359,117 +383,140 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
 
     if (warp == 0) {
-        // ---------------- TMA producer (every CTA) ----------------
-        int stage = 0;
-        uint32_t phase = 0;
-        uint32_t armed = 0;        // bit s: stage s has been armed at least once
-        uint32_t last_parity = 0;  // bit s: parity of the phase last armed on stage s
-        bool ok = true;
-        for (int tile = group; tile < num_tiles && ok; tile += num_groups) {
-            const int m0 = (tile % tiles_m) * G::TILE_M + (int)rank * G::ROWS_PER_CTA;
-            const int n0 = (tile / tiles_m) * BN + (int)rank * G::B_COLS_PER_CTA;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) {
-                    if (lane == 0) record_timeout(status, bars, 1, (unsigned)tile);
-                    break;
-                }
-                if (lane == 0) {
-                    const uint32_t own_bar = smem_u32(&bars->full[stage]);
-                    // the pair's loads are counted by the first CTA's barrier
-                    const uint32_t bar = (CTAS == 1) ? own_bar : map_to_cta(own_bar, 0);
+        // ---------------- TMA producer (one thread of every CTA) ----------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t armed = 0;        // bit s: stage s has been armed at least once
+            uint32_t last_parity = 0;  // bit s: parity of the phase last armed on stage s
+            bool ok = true;
+            const uint32_t full0 = smem_u32(&bars->full[0]);
+            // the pair's loads are counted by the first CTA's barrier
+            const uint32_t full0_lead = (CTAS == 1) ? full0 : map_to_cta(full0, 0);
+            for (int tile = group; tile < num_items && ok; tile += num_groups) {
+                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+                const int cols_per_cta = wi.width / CTAS;  // dY columns this CTA stages
+                const int b_boxes = cols_per_cta / GROUP;
+                const int m0 = wi.m0 + (int)rank * G::ROWS_PER_CTA;
+                const int n0 = wi.n0 + (int)rank * cols_per_cta;
+                const uint32_t stage_tx =
+                    (uint32_t)(G::A_STAGE_BYTES + b_boxes * BOX_BYTES) * CTAS;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
+                    if (!ok) {
+                        record_timeout(status, bars, 1, (unsigned)tile);
+                        break;
+                    }
+                    const uint32_t bar = full0_lead + (uint32_t)stage * 8u;
                     const uint32_t sa = base + stage * G::STAGE_BYTES;
                     const uint32_t sb = sa + G::A_STAGE_BYTES;
                     // out-of-range parts of a box are zero-filled and still counted
-                    if (rank == 0) mbar_arrive_expect_tx(own_bar, G::STAGE_BYTES * CTAS);
+                    if (rank == 0) mbar_arrive_expect_tx(full0 + (uint32_t)stage * 8u, stage_tx);
 #pragma unroll
                     for (int j = 0; j < G::A_BOXES; ++j)
                         tma_load_2d<CTAS>(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK, bar);
-#pragma unroll
-                    for (int j = 0; j < G::B_BOXES; ++j)
-                        tma_load_2d<CTAS>(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK, bar);
-                }
-                armed |= 1u << stage;
-                last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
-                __syncwarp();
-                if (++stage == STAGES) {
-                    stage = 0;
-                    phase ^= 1;
-                }
-            }
-        }
-        if (*abort_flag && rank == 0) {
-            // leave no copy in flight behind: wait (bounded) for every armed stage to land
-            int never = 0;
-            for (int s = 0; s < STAGES; ++s)
-                if (armed & (1u << s))
-                    mbar_wait(smem_u32(&bars->full[s]), (last_parity >> s) & 1u, &never,
-                              kDrainLimitNs);
-        }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer (first CTA of the pair only) ----------------
-        if (rank == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            int it = 0;
-            for (int tile = group; tile < num_tiles && ok; tile += num_groups, ++it) {
-                const int as = it & 1;
-                const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-                ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) {
-                    if (lane == 0) record_timeout(status, bars, 2, (unsigned)tile);
-                    break;
-                }
-                tc_fence_after();
-                const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) {
-                        if (lane == 0) record_timeout(status, bars, 3, (unsigned)tile);
-                        break;
-                    }
-                    tc_fence_after();
-                    if (lane == 0) {
-                        const uint32_t sa = base + stage * G::STAGE_BYTES;
-                        const uint32_t sb = sa + G::A_STAGE_BYTES;
-#pragma unroll
-                        for (int k = 0; k < BK / UMMA_K; ++k) {
-                            // 16 tokens further = 16 rows of 128 bytes
-                            const uint64_t da = make_smem_desc(sa + k * (UMMA_K * 128));
-                            const uint64_t db = make_smem_desc(sb + k * (UMMA_K * 128));
-                            tc_mma<CTAS>(tmem_d, da, db, G::INSTR_DESC, (kb | k) != 0 ? 1u : 0u);
-                        }
-                        // the stage is free, in every CTA of the pair, once these MMAs retire
-                        const uint32_t e = smem_u32(&bars->empty[stage]);
-#pragma unroll
-                        for (int r = 0; r < CTAS; ++r)
-                            tc_commit<CTAS>(CTAS == 1 ? e : map_to_cta(e, r));
-                    }
-                    __syncwarp();
+                    for (int j = 0; j < b_boxes; ++j)
+                        tma_load_2d<CTAS>(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK,
+                                          bar);
+                    armed |= 1u << stage;
+                    last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == STAGES) {
                         stage = 0;
                         phase ^= 1;
                     }
                 }
-                if (ok && lane == 0) {
+            }
+            if (*abort_flag && rank == 0) {
+                // leave no copy in flight behind: wait (bounded) for every armed stage to land
+                int never = 0;
+                for (int s = 0; s < STAGES; ++s)
+                    if (armed & (1u << s))
+                        mbar_wait(full0 + (uint32_t)s * 8u, (last_parity >> s) & 1u, &never,
+                                  kDrainLimitNs);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (one thread of the pair's first CTA) ----------------
+        // The tensor core runs in step with the issuing thread (few MMAs can be queued), so
+        // whatever the thread does between two MMAs is exposed.  The barrier of the NEXT
+        // stage is therefore probed while the current stage's MMAs are still executing.
+        if (rank == 0 && lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            const uint32_t desc_lo0 = smem_desc_lo(base);  // operand A of stage 0
+            const uint32_t full0 = smem_u32(&bars->full[0]);
+            uint32_t empty_bar0[CTAS];  // empty[0] in each CTA of the pair
+#pragma unroll
+            for (int r = 0; r < CTAS; ++r)
+                empty_bar0[r] = CTAS == 1 ? smem_u32(&bars->empty[0])
+                                          : map_to_cta(smem_u32(&bars->empty[0]), r);
+            bool next_ready = false;  // full[stage] already seen complete by a probe
+            for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
+                const int as = it & 1;
+                const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+                const uint32_t idesc =
+                    G::INSTR_DESC_NO_N |
+                    ((uint32_t)(work_item<CTAS>(tile, split_from, tiles_m).width >> 3) << 17);
+                ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
+                if (!ok) {
+                    record_timeout(status, bars, 2, (unsigned)tile);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!next_ready) {
+                        ok = mbar_wait(full0 + (uint32_t)stage * 8u, phase, abort_flag);
+                        if (!ok) {
+                            record_timeout(status, bars, 3, (unsigned)tile);
+                            break;
+                        }
+                    }
+                    tc_fence_after();
+                    const uint32_t a_lo = desc_lo0 + (uint32_t)stage * (G::STAGE_BYTES >> 4);
+                    const uint32_t b_lo = a_lo + (G::A_STAGE_BYTES >> 4);
+                    int nstage = stage + 1;
+                    uint32_t nphase = phase;
+                    if (nstage == STAGES) {
+                        nstage = 0;
+                        nphase ^= 1;
+                    }
+                    // 16 tokens further = 16 rows of 128 bytes
+                    constexpr uint32_t kstep = (UMMA_K * 128) >> 4;
+                    constexpr int KSTEPS = BK / UMMA_K;
+#pragma unroll
+                    for (int k = 0; k < KSTEPS - 1; ++k)
+                        tc_mma<CTAS>(tmem_d, smem_desc(a_lo + k * kstep),
+                                     smem_desc(b_lo + k * kstep), idesc, (kb | k) != 0 ? 1u : 0u);
+                    // look ahead while those execute (a stale "ready" cannot occur: the
+                    // barrier cannot advance two phases before this thread frees the stage)
+                    next_ready = mbar_try_wait(full0 + (uint32_t)nstage * 8u, nphase);
+                    tc_mma<CTAS>(tmem_d, smem_desc(a_lo + (KSTEPS - 1) * kstep),
+                                 smem_desc(b_lo + (KSTEPS - 1) * kstep), idesc, 1u);
+                    // the stage is free, in every CTA of the pair, once these MMAs retire
+#pragma unroll
+                    for (int r = 0; r < CTAS; ++r)
+                        tc_commit<CTAS>(empty_bar0[r] + (uint32_t)stage * 8u);
+                    stage = nstage;
+                    phase = nphase;
+                }
+                if (ok) {
                     const uint32_t f = smem_u32(&bars->acc_full[as]);
 #pragma unroll
                     for (int r = 0; r < CTAS; ++r) tc_commit<CTAS>(CTAS == 1 ? f : map_to_cta(f, r));
                 }
-                __syncwarp();
             }
             if (*abort_flag) {
                 // let issued MMAs retire before TMEM is given back
-                if (lane == 0) tc_commit<CTAS>(smem_u32(&bars->drain));
-                __syncwarp();
+                tc_commit<CTAS>(smem_u32(&bars->drain));
                 int never = 0;
                 mbar_wait(smem_u32(&bars->drain), 0, &never, kDrainLimitNs);
             }
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue: TMEM -> a*G, b*G^2 -> TMA reduce-add into m, v ----------
         const int q = warp & 3;  // TMEM lane quarter this warp may read
@@ -480,12 +527,12 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         const uint32_t sw = (uint32_t)(lane & 7);
         bool ok = true;
         int it = 0;
-        for (int tile = group; tile < num_tiles && ok; tile += num_groups, ++it) {
+        for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-            const int row0 =
-                (tile % tiles_m) * G::TILE_M + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
-            const int n0 = (tile / tiles_m) * BN;
+            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+            const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
+            const int n0 = wi.n0;
             ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -496,7 +543,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             if (row0 < d_in) {
                 const uint32_t taddr0 =
                     tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
-                for (int c = 0; c < BN / EPI_COLS; ++c) {
+                for (int c = 0; c < wi.width / EPI_COLS; ++c) {
                     const int col0 = n0 + c * EPI_COLS;
                     if (col0 >= d_out) break;  // boxes wholly outside the matrix are skipped
                     uint32_t r[32];
@@ -648,16 +695,24 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     }
     const int tiles_n = (p.d_out + BN - 1) / BN;
     *msg = "wgrad_fold launch";
+    const int tile_m = g_variant == 1 ? Geo<1>::TILE_M : Geo<2>::TILE_M;
+    const int tiles = ((p.d_in + tile_m - 1) / tile_m) * tiles_n;
+    const int max_groups = g_variant == 1 ? p.sm_count : p.sm_count / 2;
+    // Tail balancing: if the last round would keep at most half of the groups busy, its
+    // tiles are issued as 128-column halves (see WorkItem).
+    const int rest = tiles % max_groups;
+    int split_from = tiles, items = tiles;
+    if (rest > 0 && 2 * rest <= max_groups) {
+        split_from = tiles - rest;
+        items = tiles + rest;
+    }
+    const int groups = items < max_groups ? items : max_groups;
     if (g_variant == 1) {
-        const int tiles = ((p.d_in + Geo<1>::TILE_M - 1) / Geo<1>::TILE_M) * tiles_n;
-        const int grid = tiles < p.sm_count ? tiles : p.sm_count;
-        wgrad_fold_kernel<1><<<grid, NUM_THREADS, Geo<1>::SMEM_BYTES, p.stream>>>(
-            map_x, map_dy, map_m, map_v, p.tokens, p.d_in, p.d_out, p.c.a, p.c.b, p.status);
+        wgrad_fold_kernel<1><<<groups, NUM_THREADS, Geo<1>::SMEM_BYTES, p.stream>>>(
+            map_x, map_dy, map_m, map_v, p.tokens, p.d_in, p.d_out, split_from, items, p.c.a,
+            p.c.b, p.status);
         return cudaGetLastError();
     }
-    const int tiles = ((p.d_in + Geo<2>::TILE_M - 1) / Geo<2>::TILE_M) * tiles_n;
-    const int pairs = p.sm_count / 2;
-    const int groups = tiles < pairs ? tiles : pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
@@ -671,7 +726,7 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_m, map_v, p.tokens,
-                              p.d_in, p.d_out, p.c.a, p.c.b, p.status);
+                              p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status);
 }
 
 }  // namespace adama
