@@ -1,0 +1,96 @@
+"""Stacks of linear layers driven through the AdamA library, back to front.
+
+A `LinearStack` owns three flat fp32 device buffers (w, m, v) that hold every
+layer's [d_in, d_out] matrix back to back; each layer is a view.  One mini-batch
+follows Algorithm 2 of the AdamA paper: for every micro-batch the layers are
+visited from the last to the first (the order in which backward produces their
+gradients), each layer's (X, dY) pair is handed to the fused weight-gradient fold
+and dropped at once, and after the last micro-batch every parameter is updated.
+This module only sequences library calls and owns memory; all arithmetic is in
+the CUDA kernels.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Callable, List, Sequence, Tuple
+
+import torch
+
+from .binding import AdamA
+
+
+@dataclass(frozen=True)
+class LayerSpec:
+    name: str
+    d_in: int
+    d_out: int
+
+
+class LinearStack:
+    def __init__(self, layers: Sequence[LayerSpec], device="cuda"):
+        self.layers: List[LayerSpec] = list(layers)
+        self.device = torch.device(device)
+        self.offsets: List[int] = []
+        total = 0
+        for L in self.layers:
+            self.offsets.append(total)
+            total += L.d_in * L.d_out
+            total = (total + 63) // 64 * 64  # keep every layer 256-byte aligned
+        self.numel = total
+        self.w = torch.zeros(total, dtype=torch.float32, device=self.device)
+        self.m = torch.zeros(total, dtype=torch.float32, device=self.device)
+        self.v = torch.zeros(total, dtype=torch.float32, device=self.device)
+
+    @property
+    def n_params(self) -> int:
+        return sum(L.d_in * L.d_out for L in self.layers)
+
+    def view(self, buf: torch.Tensor, j: int) -> torch.Tensor:
+        L = self.layers[j]
+        o = self.offsets[j]
+        return buf[o:o + L.d_in * L.d_out].view(L.d_in, L.d_out)
+
+    def flops_per_micro_batch(self, tokens: int) -> float:
+        return sum(2.0 * tokens * L.d_in * L.d_out for L in self.layers)
+
+    def minibatch(self, opt: AdamA, n_micro: int, lr: float,
+                  inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]],
+                  materialise: str = "none") -> None:
+        """One mini-batch.  `inputs(micro, layer_index, spec)` returns (X, dY) for that
+        (micro-batch, layer); the tensors are released right after the layer's call.
+
+        materialise: "none"  -- fused kernel, the weight gradient never exists in memory;
+                     "layer" -- the paper's pipeline: a per-layer fp32 gradient buffer is
+                                assigned, filled by a library GEMM, folded with adama_fold
+                                and released (for memory / speed comparison only).
+        """
+        opt.begin_minibatch(n_micro)
+        for i in range(n_micro):
+            for j in reversed(range(len(self.layers))):
+                spec = self.layers[j]
+                X, dY = inputs(i, j, spec)
+                if materialise == "none":
+                    opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j))
+                else:
+                    G = torch.empty(spec.d_in, spec.d_out, dtype=torch.float32, device=self.device)
+                    torch.mm(X.t(), dY, out_dtype=torch.float32, out=G)
+                    opt.fold(G.view(-1), self.view(self.m, j).view(-1), self.view(self.v, j).view(-1))
+                    del G
+                del X, dY
+        # one apply over the whole flat buffer (padding between layers holds zeros)
+        opt.apply(self.w, self.m, self.v, lr)
+
+
+def gpt2xl_stack(blocks: int, device="cuda") -> LinearStack:
+    h = 1600
+    per_block = [("qkv", h, 3 * h), ("out_proj", h, h), ("fc1", h, 4 * h), ("fc2", 4 * h, h)]
+    return LinearStack([LayerSpec(f"b{b}.{n}", di, do) for b in range(blocks)
+                        for (n, di, do) in per_block], device)
+
+
+def llama7b_stack(blocks: int, device="cuda") -> LinearStack:
+    h, f = 4096, 11008
+    per_block = [("q", h, h), ("k", h, h), ("v", h, h), ("o", h, h),
+                 ("gate", h, f), ("up", h, f), ("down", f, h)]
+    return LinearStack([LayerSpec(f"b{b}.{n}", di, do) for b in range(blocks)
+                        for (n, di, do) in per_block], device)
