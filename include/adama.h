@@ -130,8 +130,9 @@ ADAMA_API adama_status adama_fold(adama_ctx *ctx, const void *grad, adama_dtype 
  * Any d_in, d_out, tokens within those rules are handled (ragged tiles are
  * zero-filled on load and clipped on store).  The whole token sum of one call
  * is finished before it is squared: there is no split over tokens.
- * m and v are updated by tile-wise reduce-add through the L2; each element is
- * touched exactly once per call, so results do not depend on scheduling.
+ * m and v are read, updated with one fma per element and written back by the
+ * kernel's epilogue; each element is touched by exactly one tile per call, so
+ * results do not depend on scheduling.
  * A caller that stores W as [d_out, d_in] passes (dY, X) in place of (X, dY).
  * Device-side waits are bounded; if one expires the kernel stops early, leaves
  * a code in the status block and adama_sync_status returns ADAMA_ERR_TIMEOUT.

@@ -3,10 +3,14 @@
 //   G[p,q]  = sum_tau X[tau,p] * dY[tau,q]          (bf16 x bf16 -> fp32, tcgen05.mma)
 //   m[p,q] += a*G[p,q];   v[p,q] += b*G[p,q]^2       (Algorithm 2, inner loop body)
 //
-// G lives only as an accumulator tile in tensor memory: the epilogue reads it with
-// tcgen05.ld, scales it, stages a*G and b*G^2 in shared memory and hands them to
-// the TMA unit as reduce-add stores, so m and v are read-modified-written at the
-// L2 and the SM never waits on a global load.
+// G lives only as an accumulator tile in tensor memory.  The epilogue issues the
+// coalesced 128-bit loads of the matching m and v chunk first, reads the accumulator
+// chunk with tcgen05.ld while they are in flight, turns it from "one row per thread"
+// into "128 contiguous bytes per quarter-warp" through a swizzled shared-memory
+// buffer, and writes fma(a, G, m) and fma(b*G, G, v) back with 128-bit stores.
+// (Letting the L2 do the read-modify-write -- TMA reduce-add or red.global.add.v4 --
+// was measured first: the L2's reduction rate, about 2 TB/s of payload, stalled the
+// operand loads of the overlapped main loop; plain reads and writes do not.)
 //
 // Persistent kernel, 192 threads per CTA, CTAs working in pairs (a cluster of two on
 // the two SMs of a TPC, tcgen05 cta_group::2): a pair owns a 256x256 output tile,
@@ -16,7 +20,8 @@
 // instead of 96 for a lone 128x256 tile, and leaves room for a 6-stage ring.
 //   warp 0      TMA producer: operand tiles -> shared-memory ring (both CTAs)
 //   warp 1      MMA issuer (one thread of the pair's first CTA) + TMEM allocation
-//   warps 2..5  epilogue, one TMEM lane quarter each (both CTAs)
+//   warps 2..9  epilogue: two warps per TMEM lane quarter, one per half of the tile's
+//               columns (both CTAs)
 // The 512 TMEM columns hold two 128x256 fp32 accumulators per CTA, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  (A one-CTA variant, 128x256 tiles and a
 // 4-stage ring, is kept as a template instance for comparison.)
@@ -31,7 +36,7 @@
 // Synchronisation of a pair: the first CTA's "full" barrier of a stage counts the
 // bytes of both CTAs' loads; when the MMAs that read a stage retire, tcgen05.commit
 // arrives on the "empty" barrier of each CTA; the same for accumulator-full; the
-// eight epilogue warps of the pair arrive on the first CTA's accumulator-empty
+// sixteen epilogue warps of the pair arrive on the first CTA's accumulator-empty
 // barrier.  No load uses cluster multicast.
 //
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the kernel
@@ -50,11 +55,12 @@ constexpr int BK = 64;      // tokens per pipeline stage
 constexpr int UMMA_K = 16;  // tokens per tcgen05.mma (bf16)
 constexpr int GROUP = 64;   // features per 128-byte swizzled row
 constexpr int BOX_BYTES = GROUP * BK * 2;               // 8192
-constexpr int EPI_COLS = 32;                            // fp32 columns per reduce box (128 B)
+constexpr int EPI_COLS = 32;                            // fp32 columns per epilogue chunk (128 B)
 constexpr int EPI_ROWS = 32;                            // one TMEM lane quarter
-constexpr int EPI_BUF_BYTES = EPI_ROWS * EPI_COLS * 4;  // 4096
-constexpr int EPI_WARPS = 4;
-constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
+constexpr int EPI_BUF_BYTES = EPI_ROWS * EPI_COLS * 4;  // 4096: one transposition buffer per warp
+constexpr int EPI_WARPS = 8;                            // 4 lane quarters x COL_SPLIT column parts
+constexpr int COL_SPLIT = EPI_WARPS / 4;
+constexpr int EPI_BYTES = EPI_WARPS * EPI_BUF_BYTES;
 constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
@@ -174,24 +180,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
             : "memory");
     }
 }
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int x, int y,
-                                                  uint32_t src) {
-    asm volatile(
-        "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group "
-        "[%0, {%1, %2}], [%3];" ::"l"(map),
-        "r"(x), "r"(y), "r"(src)
-        : "memory");
-}
-__device__ __forceinline__ void bulk_commit() {
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() {
-    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -275,6 +263,26 @@ __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tc_wait_ld() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr) {
+    float4 r;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "r"(addr));
+    return r;
+}
+// m and v are touched once per call: no L1 allocation
+__device__ __forceinline__ float4 ld_global_v4_stream(const float *p) {
+    float4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_global_v4(float *p, float4 x) {
+    asm volatile("st.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z),
+                 "f"(x.w)
+                 : "memory");
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, float x, float y, float z, float w) {
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z),
                  "f"(w)
@@ -340,9 +348,8 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
 template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
-                  const __grid_constant__ CUtensorMap map_dy,
-                  const __grid_constant__ CUtensorMap map_m,
-                  const __grid_constant__ CUtensorMap map_v, int tokens, int d_in, int d_out,
+                  const __grid_constant__ CUtensorMap map_dy, float *__restrict__ m_out,
+                  float *__restrict__ v_out, long long ldmv, int tokens, int d_in, int d_out,
                   int split_from, int num_items, float a, float b, unsigned *status) {
     using G = Geo<CTAS>;
     constexpr int STAGES = G::STAGES;
@@ -518,13 +525,17 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         }
         __syncwarp();
     } else {
-        // ---------------- epilogue: TMEM -> a*G, b*G^2 -> TMA reduce-add into m, v ----------
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
-        const uint32_t sm_m = base + G::SMEM_EPI_OFF + (uint32_t)q * 2 * EPI_BUF_BYTES;
-        const uint32_t sm_v = sm_m + EPI_BUF_BYTES;
-        // 128-byte swizzle: 16-byte chunk j of row r sits at chunk (j ^ (r & 7))
+        // ---------------- epilogue: m = fma(a, G, m), v = fma(b*G, G, v) ----------------
+        const int q = warp & 3;            // TMEM lane quarter this warp may read
+        const int part = (warp - 2) >> 2;  // which part of the tile's columns it handles
+        const uint32_t sm_g = base + G::SMEM_EPI_OFF + (uint32_t)(warp - 2) * EPI_BUF_BYTES;
+        // staging buffer: 32 rows of 128 bytes; 16-byte chunk j of row r sits at (j ^ (r & 7)),
+        // which makes both the row-per-thread writes and the row-segment reads conflict-free
         const uint32_t row_off = (uint32_t)lane * 128u;
         const uint32_t sw = (uint32_t)(lane & 7);
+        // coalesced side: a quarter-warp covers 128 contiguous bytes of one row
+        const int sub_row = lane >> 3;  // 0..3
+        const int c4 = lane & 7;        // which float4 of the 32-column chunk
         bool ok = true;
         int it = 0;
         for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
@@ -532,7 +543,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
             const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
             const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
-            const int n0 = wi.n0;
+            const int chunks = wi.width / (COL_SPLIT * EPI_COLS);  // chunks per warp
             ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -543,47 +554,63 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             if (row0 < d_in) {
                 const uint32_t taddr0 =
                     tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
-                for (int c = 0; c < wi.width / EPI_COLS; ++c) {
-                    const int col0 = n0 + c * EPI_COLS;
-                    if (col0 >= d_out) break;  // boxes wholly outside the matrix are skipped
+                for (int cc = 0; cc < chunks; ++cc) {
+                    const int c = part * chunks + cc;
+                    const int col0 = wi.n0 + c * EPI_COLS;
+                    if (col0 >= d_out) break;  // chunks wholly outside the matrix are skipped
+                    const long long off0 = (long long)(row0 + sub_row) * ldmv + col0 + c4 * 4;
+                    const bool interior = row0 + EPI_ROWS <= d_in && col0 + EPI_COLS <= d_out;
+                    float4 mm[8], vv[8];
+                    if (interior) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            mm[i] = ld_global_v4_stream(m_out + off0 + (long long)i * 4 * ldmv);
+                            vv[i] = ld_global_v4_stream(v_out + off0 + (long long)i * 4 * ldmv);
+                        }
+                    }
                     uint32_t r[32];
                     tc_ld_32x32(taddr0 + (uint32_t)(c * EPI_COLS), r);
                     tc_wait_ld();
-                    // first-moment increments
-                    if (lane == 0) bulk_wait_read<1>();  // previous reduce from the m buffer was read
-                    __syncwarp();
+                    __syncwarp();  // the previous chunk has been read out of the buffer
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t addr = sm_m + row_off + ((((uint32_t)j) ^ sw) << 4);
-                        st_shared_v4(addr, a * __uint_as_float(r[4 * j + 0]),
-                                     a * __uint_as_float(r[4 * j + 1]),
-                                     a * __uint_as_float(r[4 * j + 2]),
-                                     a * __uint_as_float(r[4 * j + 3]));
-                    }
-                    fence_proxy_async_smem();
+                    for (int j = 0; j < 8; ++j)
+                        st_shared_v4(sm_g + row_off + ((((uint32_t)j) ^ sw) << 4),
+                                     __uint_as_float(r[4 * j + 0]), __uint_as_float(r[4 * j + 1]),
+                                     __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
                     __syncwarp();
-                    if (lane == 0) {
-                        tma_reduce_add_2d(&map_m, col0, row0, sm_m);
-                        bulk_commit();
-                        bulk_wait_read<1>();  // previous reduce from the v buffer was read
-                    }
-                    __syncwarp();
-                    // second-moment increments
+                    if (interior) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t addr = sm_v + row_off + ((((uint32_t)j) ^ sw) << 4);
-                        const float g0 = __uint_as_float(r[4 * j + 0]);
-                        const float g1 = __uint_as_float(r[4 * j + 1]);
-                        const float g2 = __uint_as_float(r[4 * j + 2]);
-                        const float g3 = __uint_as_float(r[4 * j + 3]);
-                        st_shared_v4(addr, (b * g0) * g0, (b * g1) * g1, (b * g2) * g2,
-                                     (b * g3) * g3);
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_reduce_add_2d(&map_v, col0, row0, sm_v);
-                        bulk_commit();
+                        for (int i = 0; i < 8; ++i) {
+                            const int row = i * 4 + sub_row;
+                            const float4 g = ld_shared_v4(sm_g + (uint32_t)row * 128u +
+                                                          (uint32_t)((c4 ^ (row & 7)) << 4));
+                            mm[i].x = fmaf(a, g.x, mm[i].x);
+                            mm[i].y = fmaf(a, g.y, mm[i].y);
+                            mm[i].z = fmaf(a, g.z, mm[i].z);
+                            mm[i].w = fmaf(a, g.w, mm[i].w);
+                            vv[i].x = fmaf(b * g.x, g.x, vv[i].x);
+                            vv[i].y = fmaf(b * g.y, g.y, vv[i].y);
+                            vv[i].z = fmaf(b * g.z, g.z, vv[i].z);
+                            vv[i].w = fmaf(b * g.w, g.w, vv[i].w);
+                            st_global_v4(m_out + off0 + (long long)i * 4 * ldmv, mm[i]);
+                            st_global_v4(v_out + off0 + (long long)i * 4 * ldmv, vv[i]);
+                        }
+                    } else {
+                        // ragged edge of the matrix: element-wise, bounds-checked
+                        for (int i = 0; i < 8; ++i) {
+                            const int row = i * 4 + sub_row;
+                            if (row0 + row >= d_in) continue;
+                            const float4 g = ld_shared_v4(sm_g + (uint32_t)row * 128u +
+                                                          (uint32_t)((c4 ^ (row & 7)) << 4));
+                            const float ge[4] = {g.x, g.y, g.z, g.w};
+                            float *pm = m_out + off0 + (long long)i * 4 * ldmv;
+                            float *pv = v_out + off0 + (long long)i * 4 * ldmv;
+                            for (int e = 0; e < 4; ++e)
+                                if (col0 + c4 * 4 + e < d_out) {
+                                    pm[e] = fmaf(a, ge[e], pm[e]);
+                                    pv[e] = fmaf(b * ge[e], ge[e], pv[e]);
+                                }
+                        }
                     }
                 }
             }
@@ -596,8 +623,6 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 else mbar_arrive_cluster(map_to_cta(e, 0));
             }
         }
-        if (lane == 0) bulk_wait_all();  // reduce-adds complete before the CTA retires
-        __syncwarp();
     }
 
     tc_fence_before();
@@ -676,19 +701,13 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
         }
         g_attr_set = true;
     }
-    CUtensorMap map_x, map_dy, map_m, map_v;
+    CUtensorMap map_x, map_dy;
     bool ok = encode_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.X, (uint64_t)p.d_in,
                         (uint64_t)p.tokens, (uint64_t)p.ldx, GROUP, BK,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B) &&
               encode_2d(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.dY, (uint64_t)p.d_out,
                         (uint64_t)p.tokens, (uint64_t)p.ldy, GROUP, BK,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B) &&
-              encode_2d(&map_m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.m, (uint64_t)p.d_out,
-                        (uint64_t)p.d_in, (uint64_t)p.ldmv, EPI_COLS, EPI_ROWS,
-                        CU_TENSOR_MAP_L2_PROMOTION_NONE) &&
-              encode_2d(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.v, (uint64_t)p.d_out,
-                        (uint64_t)p.d_in, (uint64_t)p.ldmv, EPI_COLS, EPI_ROWS,
-                        CU_TENSOR_MAP_L2_PROMOTION_NONE);
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (!ok) {
         *msg = "cuTensorMapEncodeTiled rejected a tensor";
         return cudaErrorInvalidValue;
@@ -709,8 +728,8 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     const int groups = items < max_groups ? items : max_groups;
     if (g_variant == 1) {
         wgrad_fold_kernel<1><<<groups, NUM_THREADS, Geo<1>::SMEM_BYTES, p.stream>>>(
-            map_x, map_dy, map_m, map_v, p.tokens, p.d_in, p.d_out, split_from, items, p.c.a,
-            p.c.b, p.status);
+            map_x, map_dy, p.m, p.v, (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from,
+            items, p.c.a, p.c.b, p.status);
         return cudaGetLastError();
     }
     cudaLaunchConfig_t cfg = {};
@@ -725,8 +744,9 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_m, map_v, p.tokens,
-                              p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status);
+    return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, p.m, p.v,
+                              (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
+                              p.c.a, p.c.b, p.status);
 }
 
 }  // namespace adama
