@@ -153,6 +153,22 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
 ADAMA_API adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                    double lr, void *cuda_stream);
 
+/* Data-parallel variant of adama_apply (Section 3.3, Eqs. 4-7): R = world_size devices
+ * each fold their own N micro-batches into their own m and v; once per mini-batch the
+ * CALLER sums m and v over the devices (one all-reduce each, e.g. NCCL, on the same
+ * stream order); this call then takes the summed buffers and computes
+ *     m_t = m/R,  v_t = v/R^2                          (the paper's averaging of the states)
+ *     w <- w - lr * (m_t/(1-beta1^t)) / (sqrt(v_t/(1-beta2^t)) + eps)
+ *     m <- beta1*m_t,  v <- R*beta2*v_t                ("multiply v by M*beta2 instead of beta2")
+ * so that R devices x N micro-batches give exactly the update of one device with N*R
+ * micro-batches.  Every rank calls it with the same arguments and ends with the same w.
+ * Between mini-batches each rank's v therefore holds R*beta2*v_t (m holds beta1*m_t).
+ * world_size == 1 is adama_apply.  All scalings are folded, in double, into the
+ * constants of the same kernel.  Errors as adama_apply, plus INVALID_ARG (world_size < 1). */
+ADAMA_API adama_status adama_apply_allreduced(adama_ctx *ctx, float *w, float *m, float *v,
+                                              size_t n, double lr, int world_size,
+                                              void *cuda_stream);
+
 /* ---- host-buffer variants (same arithmetic, copies included) --------------------------- */
 
 /* adama_fold with the gradient in HOST memory (pinned memory for full copy
@@ -248,6 +264,12 @@ ADAMA_API int64_t adama_launch_count(const adama_ctx *ctx);
  * Errors: INVALID_ARG. */
 ADAMA_API adama_status adama_host_constants(const adama_config *cfg, int n_micro, int64_t t,
                                             double lr, float out[9]);
+
+/* The same for adama_apply_allreduced with world_size R: out[2] = lr/(1-beta1^t)/R,
+ * out[3] = 1/(1-beta2^t)/R^2, out[5..6] = beta1/R as hi + lo, out[7..8] = beta2/R as hi + lo. */
+ADAMA_API adama_status adama_host_constants_allreduced(const adama_config *cfg, int n_micro,
+                                                       int64_t t, double lr, int world_size,
+                                                       float out[9]);
 
 /* Library version, "major.minor.patch". */
 ADAMA_API const char *adama_version(void);

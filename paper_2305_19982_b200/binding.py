@@ -17,9 +17,10 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_fold_host", "adama_linear_wgrad_fold_host",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
+    "adama_host_constants_allreduced",
     "adama_version",
 ]
 
@@ -73,6 +74,9 @@ def load_library() -> ctypes.CDLL:
     L.adama_fold.argtypes = [vp, vp, ci, vp, vp, sz, vp]
     L.adama_linear_wgrad_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp]
     L.adama_apply.argtypes = [vp, vp, vp, vp, sz, dbl, vp]
+    L.adama_apply_allreduced.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
+    L.adama_host_constants_allreduced.argtypes = [ctypes.POINTER(_Config), ci, i64, dbl, ci,
+                                                  ctypes.POINTER(ctypes.c_float)]
     L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
     L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
     L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
@@ -94,12 +98,13 @@ def load_library() -> ctypes.CDLL:
     return L
 
 
-def host_constants(beta1, beta2, eps, n_micro, t, lr, flags=0):
-    """adama_host_constants: the nine fp32 constants the kernels receive (no GPU needed)."""
+def host_constants(beta1, beta2, eps, n_micro, t, lr, flags=0, world_size=1):
+    """adama_host_constants[_allreduced]: the nine fp32 constants the kernels receive (no GPU
+    needed)."""
     L = load_library()
     cfg = _Config(beta1, beta2, eps, 0, flags)
     out = (ctypes.c_float * 9)()
-    st = L.adama_host_constants(ctypes.byref(cfg), n_micro, t, lr, out)
+    st = L.adama_host_constants_allreduced(ctypes.byref(cfg), n_micro, t, lr, world_size, out)
     if st != 0:
         raise AdamAError(st, "adama_host_constants")
     return [float(x) for x in out]
@@ -207,6 +212,19 @@ class AdamA:
                                         _dev_ptr(m, torch.float32, "m"),
                                         _dev_ptr(v, torch.float32, "v"), n, float(lr),
                                         _stream_ptr(self.device)))
+
+    def apply_allreduced(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float,
+                         world_size: int) -> None:
+        """adama_apply_allreduced: m, v hold the sums over `world_size` data-parallel ranks."""
+        if not (w.is_contiguous() and m.is_contiguous() and v.is_contiguous()):
+            raise ValueError("apply needs contiguous tensors")
+        n = w.numel()
+        if m.numel() != n or v.numel() != n:
+            raise ValueError("w, m, v must have the same number of elements")
+        self._check(self._L.adama_apply_allreduced(
+            self._h, _dev_ptr(w, torch.float32, "w"), _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), n, float(lr), int(world_size),
+            _stream_ptr(self.device)))
 
     # -- host-buffer variants ---------------------------------------------------------------
     def fold_host(self, grad_host: torch.Tensor, m: torch.Tensor, v: torch.Tensor,

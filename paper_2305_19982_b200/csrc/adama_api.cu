@@ -35,15 +35,19 @@ static void split_hi_lo(double x, float *hi, float *lo) {
     *lo = (float)(x - (double)*hi);
 }
 
-ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr) {
+ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr,
+                                    int world) {
     ApplyConstants c;
+    const double R = (double)world;
     double bc1 = 1.0 - pow(beta1, (double)t);
     double bc2 = 1.0 - pow(beta2, (double)t);
-    c.step = (float)(lr / bc1);
-    c.inv_bc2 = (float)(1.0 / bc2);
+    // m_t = m/R, v_t = v/R^2 (Eqs. 6-7); w -= lr * (m_t/bc1) / (sqrt(v_t/bc2) + eps)
+    c.step = (float)(lr / bc1 / R);
+    c.inv_bc2 = (float)(1.0 / bc2 / (R * R));
     c.eps = (float)eps;
-    split_hi_lo(beta1, &c.beta1_hi, &c.beta1_lo);
-    split_hi_lo(beta2, &c.beta2_hi, &c.beta2_lo);
+    // stored for the next mini-batch: beta1*m_t = (beta1/R)*m and R*beta2*v_t = (beta2/R)*v
+    split_hi_lo(beta1 / R, &c.beta1_hi, &c.beta1_lo);
+    split_hi_lo(beta2 / R, &c.beta2_hi, &c.beta2_lo);
     return c;
 }
 
@@ -240,19 +244,30 @@ adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *
     return ADAMA_OK;
 }
 
-adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
-                         void *cuda_stream) {
+static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
+                               int world, void *cuda_stream) {
     adama_status st = check_apply_args(ctx, w, m, v, n, lr);
     if (st != ADAMA_OK) return st;
+    if (world < 1) return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply: world_size must be >= 1");
     if (n == 0) return ADAMA_OK;
     DeviceGuard guard(ctx->cfg.device);
-    adama::ApplyConstants c =
-        adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr);
+    adama::ApplyConstants c = adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2,
+                                                          ctx->cfg.eps, ctx->t, lr, world);
     cudaError_t e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
                                         static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "apply launch", e);
     ctx->launches += 1;
     return ADAMA_OK;
+}
+
+adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
+                         void *cuda_stream) {
+    return apply_impl(ctx, w, m, v, n, lr, 1, cuda_stream);
+}
+
+adama_status adama_apply_allreduced(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
+                                    double lr, int world_size, void *cuda_stream) {
+    return apply_impl(ctx, w, m, v, n, lr, world_size, cuda_stream);
 }
 
 // ---- host-buffer variants -------------------------------------------------------------------
@@ -384,9 +399,16 @@ int64_t adama_launch_count(const adama_ctx *ctx) { return ctx ? ctx->launches : 
 
 adama_status adama_host_constants(const adama_config *cfg, int n_micro, int64_t t, double lr,
                                   float out[9]) {
-    if (!config_ok(cfg) || !out || n_micro < 1 || t < 1) return ADAMA_ERR_INVALID_ARG;
+    return adama_host_constants_allreduced(cfg, n_micro, t, lr, 1, out);
+}
+
+adama_status adama_host_constants_allreduced(const adama_config *cfg, int n_micro, int64_t t,
+                                             double lr, int world_size, float out[9]) {
+    if (!config_ok(cfg) || !out || n_micro < 1 || t < 1 || world_size < 1)
+        return ADAMA_ERR_INVALID_ARG;
     adama::FoldConstants f = adama::make_fold_constants(cfg->beta1, cfg->beta2, n_micro, cfg->flags);
-    adama::ApplyConstants c = adama::make_apply_constants(cfg->beta1, cfg->beta2, cfg->eps, t, lr);
+    adama::ApplyConstants c =
+        adama::make_apply_constants(cfg->beta1, cfg->beta2, cfg->eps, t, lr, world_size);
     out[0] = f.a;
     out[1] = f.b;
     out[2] = c.step;

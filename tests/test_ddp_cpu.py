@@ -1,0 +1,112 @@
+"""Data-parallel AdamA (Section 3.3, Eqs. 4-7) without a GPU.
+
+The CUDA kernels cannot run here, so the ranks (real processes, gloo backend, world size 2)
+carry fp32 CPU states and apply the library's own host-derived constants with numpy in place
+of the kernels; what is under test is the multi-process protocol: the collective helper, the
+R*beta2 pre-scaling, the 1/R and 1/R^2 folded into the constants, and that every rank ends
+with the single-device result for N*R micro-batches (fp64 oracle)."""
+import json
+import os
+import socket
+import subprocess
+import sys
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import paper_2305_19982_b200 as adama
+from oracle import AdamAOracle
+from paper_2305_19982_b200 import ddp
+from parity import rel_l2
+
+ROOT = Path(__file__).resolve().parent.parent
+B1, B2, EPS, LR = 0.9, 0.999, 1e-8, 1e-3
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def test_allreduced_constants_fold_the_world_size():
+    R, N, t = 4, 3, 7
+    c1 = adama.host_constants(B1, B2, EPS, N, t, LR)
+    cR = adama.host_constants(B1, B2, EPS, N, t, LR, world_size=R)
+    f32 = lambda x: float(np.float32(x))
+    assert cR[0] == c1[0] and cR[1] == c1[1]            # folds are rank-local: unchanged
+    assert cR[2] == f32(LR / (1 - B1 ** t) / R)
+    assert cR[3] == f32(1 / (1 - B2 ** t) / R ** 2)
+    assert abs((cR[5] + cR[6]) - B1 / R) < 1e-14
+    assert abs((cR[7] + cR[8]) - B2 / R) < 1e-14
+    with pytest.raises(adama.AdamAError):
+        adama.host_constants(B1, B2, EPS, N, t, LR, world_size=0)
+
+
+def _rank_main(rank, world, port, n, N, steps, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(123)
+    w = rng.normal(0, 0.02, n).astype(np.float32)        # same on every rank
+    grads = rng.normal(0, 1e-2, (steps, world, N, n)).astype(np.float32)
+    m = torch.zeros(n)
+    v = torch.zeros(n)
+    f = np.float32
+    for step in range(steps):
+        t = step + 1
+        c = [f(x) for x in adama.host_constants(B1, B2, EPS, N, t, LR, world_size=world)]
+        for i in range(N):                               # rank-local folds (what adama_fold does)
+            g = grads[step, rank, i]
+            m += torch.from_numpy(c[0] * g)
+            v += torch.from_numpy((c[1] * g) * g)
+        assert ddp.allreduce_states(m, v) == world       # the one exchange per mini-batch
+        mn, vn = m.numpy(), v.numpy()
+        w = (w - c[2] * mn / (np.sqrt(vn * c[3]) + c[4])).astype(np.float32)
+        m = torch.from_numpy((mn * c[5] + mn * c[6]).astype(np.float32))
+        v = torch.from_numpy((vn * c[7] + vn * c[8]).astype(np.float32))
+    np.savez(Path(out_dir) / f"rank{rank}.npz", w=w, m=m.numpy(), v=v.numpy())
+    dist.destroy_process_group()
+
+
+def test_two_ranks_equal_one_device_with_NR_micro_batches(tmp_path):
+    world, n, N, steps = 2, 64, 3, 3
+    port = _free_port()
+    mp.spawn(_rank_main, args=(world, port, n, N, steps, str(tmp_path)), nprocs=world, join=True)
+    rng = np.random.default_rng(123)
+    w0 = rng.normal(0, 0.02, n).astype(np.float32)
+    grads = rng.normal(0, 1e-2, (steps, world, N, n)).astype(np.float32)
+    orc = AdamAOracle(w0.astype(np.float64), B1, B2, EPS)
+    for step in range(steps):
+        orc.begin_minibatch(N * world)
+        for r in range(world):
+            for i in range(N):
+                # each rank scales by its local N, then the states are averaged over R ranks
+                orc.fold(grads[step, r, i].astype(np.float64))
+        orc.update(LR)
+    res = [np.load(tmp_path / f"rank{r}.npz") for r in range(world)]
+    for r in range(world):
+        assert rel_l2(res[r]["w"], orc.theta) <= 1e-6
+        assert rel_l2(res[r]["m"], B1 * orc.m) <= 1e-6
+        assert rel_l2(res[r]["v"], world * B2 * orc.v) <= 1e-6      # pre-scaled for the next step
+    assert np.array_equal(res[0]["w"], res[1]["w"])
+
+
+def test_bench_reference_arm_under_torchrun_prints_one_line():
+    """Multi-rank launch contract: rank 0 alone runs and prints, the others exit 0."""
+    port = _free_port()
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    out = subprocess.run(
+        [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+         "--master-addr", "127.0.0.1", "--master-port", str(port), str(ROOT / "bench.py"),
+         "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0"],
+        capture_output=True, text=True, timeout=600, env=env, cwd=str(ROOT))
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"

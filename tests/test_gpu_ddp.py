@@ -1,0 +1,81 @@
+"""adama_apply_allreduced on one GPU: R data-parallel ranks are emulated one after the other
+with separate state buffers (no kernels waiting on each other), their m and v are summed with
+a torch add standing in for the all-reduce, and every rank applies.  Section 3.3, Eqs. 4-7:
+the result must equal single-device AdamA with N*R micro-batches (fp64 oracle)."""
+import pytest
+import torch
+
+import adama_workloads as wl
+import paper_2305_19982_b200 as adama
+from oracle import AdamADDPOracle, AdamAOracle
+from parity import f64, rel_l2
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-6
+
+
+@pytest.mark.parametrize("R,N", [(2, 3), (4, 2), (8, 1)])
+def test_allreduced_apply_equals_single_device(R, N):
+    n, steps = 100_003, 3
+    w0 = wl.normal((n,), 0.02, torch.float32, 1)
+    single = AdamAOracle(f64(w0))
+    ddp_orc = AdamADDPOracle(f64(w0), R)
+    opts = [adama.AdamA() for _ in range(R)]
+    w = [w0.cuda() for _ in range(R)]
+    m = [torch.zeros(n, device="cuda") for _ in range(R)]
+    v = [torch.zeros(n, device="cuda") for _ in range(R)]
+    for step in range(steps):
+        single.begin_minibatch(N * R)
+        ddp_orc.begin_minibatch(N)
+        for r in range(R):
+            opts[r].begin_minibatch(N)
+            for i in range(N):
+                g = wl.normal((n,), 1e-2, torch.float32, 1000 * step + 10 * r + i + 7)
+                opts[r].fold(g.cuda(), m[r], v[r])
+                single.fold(f64(g))
+                ddp_orc.fold(r, f64(g))
+        m_sum = torch.stack(m).sum(0)          # stands in for all-reduce(SUM)
+        v_sum = torch.stack(v).sum(0)
+        for r in range(R):
+            m[r].copy_(m_sum)
+            v[r].copy_(v_sum)
+            opts[r].apply_allreduced(w[r], m[r], v[r], wl.LR, R)
+        single.update(wl.LR)
+        ddp_orc.allreduce_and_update(wl.LR)
+        for r in range(R):
+            assert rel_l2(f64(w[r]), single.theta) <= TOL
+            assert rel_l2(f64(w[r]), ddp_orc.theta) <= TOL
+            assert rel_l2(f64(m[r]), wl.BETA1 * single.m) <= TOL
+            assert rel_l2(f64(v[r]), R * wl.BETA2 * single.v) <= TOL
+        assert all(torch.equal(w[0], w[r]) for r in range(1, R))
+    for o in opts:
+        o.close()
+
+
+def test_world_size_one_is_plain_apply():
+    n = 4099
+    g = wl.normal((n,), 1e-2, torch.float32, 3).cuda()
+    res = []
+    for ddp in (False, True):
+        opt = adama.AdamA()
+        opt.begin_minibatch(1)
+        w = wl.normal((n,), 0.02, torch.float32, 4).cuda()
+        m, v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+        opt.fold(g, m, v)
+        if ddp:
+            opt.apply_allreduced(w, m, v, wl.LR, 1)
+        else:
+            opt.apply(w, m, v, wl.LR)
+        res.append((w.clone(), m.clone(), v.clone()))
+        opt.close()
+    assert all(torch.equal(a, b) for a, b in zip(*res))
+
+
+def test_world_size_must_be_positive():
+    opt = adama.AdamA()
+    opt.begin_minibatch(1)
+    x = torch.zeros(8, device="cuda")
+    with pytest.raises(adama.AdamAError) as e:
+        opt.apply_allreduced(x, x.clone(), x.clone(), 1e-3, 0)
+    assert e.value.status == adama.Status.ERR_INVALID_ARG
+    opt.close()
