@@ -169,6 +169,21 @@ ADAMA_API adama_status adama_apply_allreduced(adama_ctx *ctx, float *w, float *m
                                               size_t n, double lr, int world_size,
                                               void *cuda_stream);
 
+/* State-sharded variant: the paper combines AdamA with ZeRO-DP P_os (Section 4.2, "Memory
+ * Reduction") but prints no algorithm for it; this is this library's construction on top of
+ * Section 3.3, chosen so that Eqs. 6-7 still hold.  Rank r owns one contiguous shard of every parameter buffer.  Each rank still
+ * folds full-size local accumulators m, v; once per mini-batch the CALLER reduce-scatters
+ * (sums) them so that the owner holds the summed shard, calls this function on its shard of
+ * w, m, v, zero-fills the shards of m and v it does not own, and all-gathers w.  With
+ * S_m, S_v the summed shard:
+ *     m_t = S_m/R,  v_t = S_v/R^2,  w <- w - lr * (m_t/(1-beta1^t)) / (sqrt(v_t/(1-beta2^t)) + eps)
+ *     m <- beta1*S_m (= R*beta1*m_t),  v <- beta2*S_v (= R^2*beta2*v_t)
+ * The un-normalised storage is what makes the next mini-batch's sum come out right when the
+ * non-owners restart from zero: (beta2*S_v + new folds)/R^2 = beta2*v_t + ... (Eq. 7).
+ * Persistent optimizer state per rank is 1/R of m and v.  Errors as adama_apply_allreduced. */
+ADAMA_API adama_status adama_apply_sharded(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
+                                           double lr, int world_size, void *cuda_stream);
+
 /* ---- host-buffer variants (same arithmetic, copies included) --------------------------- */
 
 /* adama_fold with the gradient in HOST memory (pinned memory for full copy
@@ -270,6 +285,12 @@ ADAMA_API adama_status adama_host_constants(const adama_config *cfg, int n_micro
 ADAMA_API adama_status adama_host_constants_allreduced(const adama_config *cfg, int n_micro,
                                                        int64_t t, double lr, int world_size,
                                                        float out[9]);
+
+/* The same for adama_apply_sharded: as _allreduced, but out[5..6] = beta1 and out[7..8] = beta2
+ * (hi + lo), since the owner keeps the un-normalised sums. */
+ADAMA_API adama_status adama_host_constants_sharded(const adama_config *cfg, int n_micro,
+                                                    int64_t t, double lr, int world_size,
+                                                    float out[9]);
 
 /* Library version, "major.minor.patch". */
 ADAMA_API const char *adama_version(void);

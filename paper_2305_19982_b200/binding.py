@@ -17,10 +17,10 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_fold_host", "adama_linear_wgrad_fold_host",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
-    "adama_host_constants_allreduced",
+    "adama_host_constants_allreduced", "adama_host_constants_sharded",
     "adama_version",
 ]
 
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     L.adama_apply_allreduced.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
     L.adama_host_constants_allreduced.argtypes = [ctypes.POINTER(_Config), ci, i64, dbl, ci,
                                                   ctypes.POINTER(ctypes.c_float)]
+    L.adama_apply_sharded.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
+    L.adama_host_constants_sharded.argtypes = L.adama_host_constants_allreduced.argtypes
     L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
     L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
     L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
@@ -98,13 +100,14 @@ def load_library() -> ctypes.CDLL:
     return L
 
 
-def host_constants(beta1, beta2, eps, n_micro, t, lr, flags=0, world_size=1):
-    """adama_host_constants[_allreduced]: the nine fp32 constants the kernels receive (no GPU
-    needed)."""
+def host_constants(beta1, beta2, eps, n_micro, t, lr, flags=0, world_size=1, sharded=False):
+    """adama_host_constants[_allreduced|_sharded]: the nine fp32 constants the kernels receive
+    (no GPU needed)."""
     L = load_library()
     cfg = _Config(beta1, beta2, eps, 0, flags)
     out = (ctypes.c_float * 9)()
-    st = L.adama_host_constants_allreduced(ctypes.byref(cfg), n_micro, t, lr, world_size, out)
+    fn = L.adama_host_constants_sharded if sharded else L.adama_host_constants_allreduced
+    st = fn(ctypes.byref(cfg), n_micro, t, lr, world_size, out)
     if st != 0:
         raise AdamAError(st, "adama_host_constants")
     return [float(x) for x in out]
@@ -222,6 +225,20 @@ class AdamA:
         if m.numel() != n or v.numel() != n:
             raise ValueError("w, m, v must have the same number of elements")
         self._check(self._L.adama_apply_allreduced(
+            self._h, _dev_ptr(w, torch.float32, "w"), _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), n, float(lr), int(world_size),
+            _stream_ptr(self.device)))
+
+    def apply_sharded(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float,
+                      world_size: int) -> None:
+        """adama_apply_sharded: w, m, v are this rank's shard; m, v hold the reduce-scattered
+        sums over `world_size` ranks."""
+        if not (w.is_contiguous() and m.is_contiguous() and v.is_contiguous()):
+            raise ValueError("apply needs contiguous tensors")
+        n = w.numel()
+        if m.numel() != n or v.numel() != n:
+            raise ValueError("w, m, v must have the same number of elements")
+        self._check(self._L.adama_apply_sharded(
             self._h, _dev_ptr(w, torch.float32, "w"), _dev_ptr(m, torch.float32, "m"),
             _dev_ptr(v, torch.float32, "v"), n, float(lr), int(world_size),
             _stream_ptr(self.device)))

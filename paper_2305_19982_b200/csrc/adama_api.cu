@@ -36,7 +36,7 @@ static void split_hi_lo(double x, float *hi, float *lo) {
 }
 
 ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr,
-                                    int world) {
+                                    int world, bool sharded) {
     ApplyConstants c;
     const double R = (double)world;
     double bc1 = 1.0 - pow(beta1, (double)t);
@@ -46,8 +46,9 @@ ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int6
     c.inv_bc2 = (float)(1.0 / bc2 / (R * R));
     c.eps = (float)eps;
     // stored for the next mini-batch: beta1*m_t = (beta1/R)*m and R*beta2*v_t = (beta2/R)*v
-    split_hi_lo(beta1 / R, &c.beta1_hi, &c.beta1_lo);
-    split_hi_lo(beta2 / R, &c.beta2_hi, &c.beta2_lo);
+    // (sharded: the owner keeps R*beta1*m_t = beta1*m and R^2*beta2*v_t = beta2*v)
+    split_hi_lo(sharded ? beta1 : beta1 / R, &c.beta1_hi, &c.beta1_lo);
+    split_hi_lo(sharded ? beta2 : beta2 / R, &c.beta2_hi, &c.beta2_lo);
     return c;
 }
 
@@ -245,14 +246,14 @@ adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *
 }
 
 static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
-                               int world, void *cuda_stream) {
+                               int world, bool sharded, void *cuda_stream) {
     adama_status st = check_apply_args(ctx, w, m, v, n, lr);
     if (st != ADAMA_OK) return st;
     if (world < 1) return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply: world_size must be >= 1");
     if (n == 0) return ADAMA_OK;
     DeviceGuard guard(ctx->cfg.device);
     adama::ApplyConstants c = adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2,
-                                                          ctx->cfg.eps, ctx->t, lr, world);
+                                                          ctx->cfg.eps, ctx->t, lr, world, sharded);
     cudaError_t e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
                                         static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "apply launch", e);
@@ -262,12 +263,17 @@ static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, siz
 
 adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
                          void *cuda_stream) {
-    return apply_impl(ctx, w, m, v, n, lr, 1, cuda_stream);
+    return apply_impl(ctx, w, m, v, n, lr, 1, false, cuda_stream);
 }
 
 adama_status adama_apply_allreduced(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                     double lr, int world_size, void *cuda_stream) {
-    return apply_impl(ctx, w, m, v, n, lr, world_size, cuda_stream);
+    return apply_impl(ctx, w, m, v, n, lr, world_size, false, cuda_stream);
+}
+
+adama_status adama_apply_sharded(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
+                                 int world_size, void *cuda_stream) {
+    return apply_impl(ctx, w, m, v, n, lr, world_size, true, cuda_stream);
 }
 
 // ---- host-buffer variants -------------------------------------------------------------------
@@ -400,6 +406,19 @@ int64_t adama_launch_count(const adama_ctx *ctx) { return ctx ? ctx->launches : 
 adama_status adama_host_constants(const adama_config *cfg, int n_micro, int64_t t, double lr,
                                   float out[9]) {
     return adama_host_constants_allreduced(cfg, n_micro, t, lr, 1, out);
+}
+
+adama_status adama_host_constants_sharded(const adama_config *cfg, int n_micro, int64_t t, double lr,
+                                          int world_size, float out[9]) {
+    adama_status st = adama_host_constants_allreduced(cfg, n_micro, t, lr, world_size, out);
+    if (st != ADAMA_OK) return st;
+    adama::ApplyConstants c =
+        adama::make_apply_constants(cfg->beta1, cfg->beta2, cfg->eps, t, lr, world_size, true);
+    out[5] = c.beta1_hi;
+    out[6] = c.beta1_lo;
+    out[7] = c.beta2_hi;
+    out[8] = c.beta2_lo;
+    return ADAMA_OK;
 }
 
 adama_status adama_host_constants_allreduced(const adama_config *cfg, int n_micro, int64_t t,

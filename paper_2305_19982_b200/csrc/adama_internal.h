@@ -31,8 +31,11 @@ FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsig
 // world > 1: m and v hold the SUM over `world` data-parallel ranks (Section 3.3 of the paper);
 // the 1/world and 1/world^2 of Eqs. 6-7 and the world*beta2 pre-scaling of the next mini-batch
 // are folded into the same constants, so the kernel is unchanged.
+// sharded (ZeRO-style ownership): the caller's m, v are the owner's shard of the summed
+// states and stay un-normalised between mini-batches (beta*sum instead of beta/R*sum),
+// because the other ranks restart their accumulators for that shard from zero.
 ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr,
-                                    int world = 1);
+                                    int world = 1, bool sharded = false);
 
 // Status block in device memory (256 bytes): word 0 = first error code recorded
 // by a kernel (0 = none), word 1 = which wait, word 2 = tile; rest reserved.

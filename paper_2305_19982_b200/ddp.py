@@ -25,3 +25,44 @@ def allreduce_and_apply(opt, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, 
     """End of a mini-batch on every rank: one state all-reduce, then the fused update."""
     world = allreduce_states(m, v, group)
     opt.apply_allreduced(w, m, v, lr, world)
+
+
+def shard_bounds(n: int, world: int, rank: int):
+    """Contiguous equal shards; n must be a multiple of world (pad the flat buffer)."""
+    if n % world:
+        raise ValueError("buffer length must be a multiple of the world size")
+    k = n // world
+    return rank * k, (rank + 1) * k
+
+
+def reduce_scatter_states(m: torch.Tensor, v: torch.Tensor, group=None):
+    """Sums m and v over the ranks so that this rank's own shard holds the sum (in place);
+    returns (lo, hi, world).  Backends without reduce-scatter fall back to an all-reduce."""
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    lo, hi = shard_bounds(m.numel(), world, rank)
+    for buf in (m, v):
+        flat = buf.view(-1)
+        try:
+            dist.reduce_scatter_tensor(flat[lo:hi], flat, op=dist.ReduceOp.SUM, group=group)
+        except (RuntimeError, NotImplementedError):
+            dist.all_reduce(flat, op=dist.ReduceOp.SUM, group=group)
+    return lo, hi, world
+
+
+def reduce_scatter_apply_allgather(opt, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
+                                   lr: float, group=None) -> None:
+    """End of a mini-batch with sharded optimizer states: reduce-scatter m, v; the owner
+    updates its shard of w; shards of m, v owned by other ranks restart from zero; all-gather w."""
+    lo, hi, world = reduce_scatter_states(m, v, group)
+    wf, mf, vf = w.view(-1), m.view(-1), v.view(-1)
+    opt.apply_sharded(wf[lo:hi], mf[lo:hi], vf[lo:hi], lr, world)
+    mf[:lo].zero_()
+    mf[hi:].zero_()
+    vf[:lo].zero_()
+    vf[hi:].zero_()
+    try:
+        dist.all_gather_into_tensor(wf, wf[lo:hi].clone(), group=group)
+    except (RuntimeError, NotImplementedError):
+        parts = [torch.empty_like(wf[lo:hi]) for _ in range(world)]
+        dist.all_gather(parts, wf[lo:hi].clone(), group=group)
+        wf.copy_(torch.cat(parts))

@@ -96,6 +96,72 @@ def test_two_ranks_equal_one_device_with_NR_micro_batches(tmp_path):
     assert np.array_equal(res[0]["w"], res[1]["w"])
 
 
+def _sharded_rank_main(rank, world, port, n, N, steps, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(321)
+    w = torch.from_numpy(rng.normal(0, 0.02, n).astype(np.float32))
+    grads = rng.normal(0, 1e-2, (steps, world, N, n)).astype(np.float32)
+    m = torch.zeros(n)
+    v = torch.zeros(n)
+    f = np.float32
+
+    class NumpyApply:                      # stands in for the CUDA kernel, same constants
+        def __init__(self):
+            self.t = 0
+
+        def apply_sharded(self, ws, ms, vs, lr, R):
+            c = [f(x) for x in adama.host_constants(B1, B2, EPS, N, self.t, lr, world_size=R,
+                                                    sharded=True)]
+            mn, vn = ms.numpy().copy(), vs.numpy().copy()
+            ws.copy_(torch.from_numpy((ws.numpy() - c[2] * mn / (np.sqrt(vn * c[3]) + c[4])).astype(f)))
+            ms.copy_(torch.from_numpy((mn * c[5] + mn * c[6]).astype(f)))
+            vs.copy_(torch.from_numpy((vn * c[7] + vn * c[8]).astype(f)))
+
+    opt = NumpyApply()
+    for step in range(steps):
+        opt.t = step + 1
+        a, b = [f(x) for x in adama.host_constants(B1, B2, EPS, N, opt.t, LR)[:2]]
+        for i in range(N):
+            g = grads[step, rank, i]
+            m += torch.from_numpy(a * g)
+            v += torch.from_numpy((b * g) * g)
+        ddp.reduce_scatter_apply_allgather(opt, w, m, v, LR)
+    lo, hi = ddp.shard_bounds(n, world, rank)
+    np.savez(Path(out_dir) / f"shard{rank}.npz", w=w.numpy(), m=m.numpy(), v=v.numpy(), lo=lo, hi=hi)
+    dist.destroy_process_group()
+
+
+def test_sharded_states_two_ranks_equal_one_device(tmp_path):
+    """Reduce-scatter, owner-only update with un-normalised storage, zeroed foreign shards,
+    all-gather of w: same weights as one device with N*R micro-batches, and each rank keeps
+    persistent state only for its own shard."""
+    world, n, N, steps = 2, 64, 2, 3
+    port = _free_port()
+    mp.spawn(_sharded_rank_main, args=(world, port, n, N, steps, str(tmp_path)), nprocs=world,
+             join=True)
+    rng = np.random.default_rng(321)
+    w0 = rng.normal(0, 0.02, n).astype(np.float32)
+    grads = rng.normal(0, 1e-2, (steps, world, N, n)).astype(np.float32)
+    orc = AdamAOracle(w0.astype(np.float64), B1, B2, EPS)
+    for step in range(steps):
+        orc.begin_minibatch(N * world)
+        for r in range(world):
+            for i in range(N):
+                orc.fold(grads[step, r, i].astype(np.float64))
+        orc.update(LR)
+    for r in range(world):
+        d = np.load(tmp_path / f"shard{r}.npz")
+        lo, hi = int(d["lo"]), int(d["hi"])
+        assert rel_l2(d["w"], orc.theta) <= 1e-6                       # full weights everywhere
+        assert rel_l2(d["m"][lo:hi], world * B1 * orc.m[lo:hi]) <= 1e-6
+        assert rel_l2(d["v"][lo:hi], world ** 2 * B2 * orc.v[lo:hi]) <= 1e-6
+        other = np.ones(n, bool)
+        other[lo:hi] = False
+        assert not d["m"][other].any() and not d["v"][other].any()
+
+
 def test_bench_reference_arm_under_torchrun_prints_one_line():
     """Multi-rank launch contract: rank 0 alone runs and prints, the others exit 0."""
     port = _free_port()

@@ -79,3 +79,43 @@ def test_world_size_must_be_positive():
         opt.apply_allreduced(x, x.clone(), x.clone(), 1e-3, 0)
     assert e.value.status == adama.Status.ERR_INVALID_ARG
     opt.close()
+
+
+@pytest.mark.parametrize("R,N", [(2, 2), (4, 1)])
+def test_sharded_apply_equals_single_device(R, N):
+    """adama_apply_sharded with R ranks emulated in turn: full-size local accumulators, summed
+    shard by shard (standing in for reduce-scatter), owner-only update, foreign shards zeroed,
+    weights gathered."""
+    n, steps = 8 * 4099, 3
+    k = n // R
+    w0 = wl.normal((n,), 0.02, torch.float32, 11)
+    single = AdamAOracle(f64(w0))
+    opts = [adama.AdamA() for _ in range(R)]
+    w = w0.cuda()                                     # identical on all ranks after the gather
+    m = [torch.zeros(n, device="cuda") for _ in range(R)]
+    v = [torch.zeros(n, device="cuda") for _ in range(R)]
+    for step in range(steps):
+        single.begin_minibatch(N * R)
+        for r in range(R):
+            opts[r].begin_minibatch(N)
+            for i in range(N):
+                g = wl.normal((n,), 1e-2, torch.float32, 2000 * step + 10 * r + i + 3)
+                opts[r].fold(g.cuda(), m[r], v[r])
+                single.fold(f64(g))
+        m_sum = torch.stack(m).sum(0)
+        v_sum = torch.stack(v).sum(0)
+        for r in range(R):
+            lo, hi = r * k, (r + 1) * k
+            m[r].zero_()
+            v[r].zero_()
+            m[r][lo:hi] = m_sum[lo:hi]
+            v[r][lo:hi] = v_sum[lo:hi]
+            opts[r].apply_sharded(w[lo:hi], m[r][lo:hi], v[r][lo:hi], wl.LR, R)
+        single.update(wl.LR)
+        assert rel_l2(f64(w), single.theta) <= TOL
+        for r in range(R):
+            lo, hi = r * k, (r + 1) * k
+            assert rel_l2(f64(m[r][lo:hi]), R * wl.BETA1 * single.m[lo:hi]) <= TOL
+            assert rel_l2(f64(v[r][lo:hi]), R * R * wl.BETA2 * single.v[lo:hi]) <= TOL
+    for o in opts:
+        o.close()
