@@ -2,7 +2,7 @@
 """Benchmark of the AdamA hot path on B200: fold / apply GB/s and fused wgrad+fold TFLOP/s.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload headline|gpt2xl|llama7b]
+                    [--workload headline|gpt2xl|llama7b|sweep]
 
 One step of the headline workload = one pass of the whole path:
   phase A  (flat 335M-parameter buffer, bf16 gradients, N=8):
@@ -574,6 +574,51 @@ def run_stack(args):
     opt.close()
 
 
+def run_sweep(args):
+    """Config 2's size sweep: fold (bf16 g) and apply at 2^20 .. 2^28 and 335 M elements;
+    median and best of 30 launches each, L2 flushed before every launch for sizes that
+    would otherwise stay L2-resident."""
+    import paper_2305_19982_b200 as adama
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pk = peaks()
+    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
+    opt.begin_minibatch(wl.CONFIG2.n_micro)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    rows = []
+    for n in wl.CONFIG2_SWEEP:
+        w = wl.normal((n,), 0.02, torch.float32, 1, device=dev)
+        m = torch.zeros(n, device=dev)
+        v = torch.zeros(n, device=dev)
+        g = wl.normal((n,), wl.CONFIG2.grad_std, torch.bfloat16, 2, device=dev)
+        res = {"n": n}
+        for name, call, bpp in (("fold", lambda: opt.fold(g, m, v), FOLD_BYTES_BF16),
+                                ("apply", lambda: opt.apply(w, m, v, wl.LR), APPLY_BYTES)):
+            for _ in range(3):
+                call()
+            ts = []
+            for _ in range(30):
+                flush.zero_()
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+                call()
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            ts.sort()
+            med, best = ts[len(ts) // 2], ts[0]
+            res[name] = {"us_median": med * 1e3, "us_best": best * 1e3,
+                         "GBps_median": bpp * n / (med * 1e-3) / 1e9,
+                         "frac_of_peak": bpp * n / (med * 1e-3) / 1e9 / pk["hbm_gbs"]}
+        rows.append(res)
+        del w, m, v, g
+    print(json.dumps({"metric": "adama_fold_apply_size_sweep", "unit": "GB/s", "peak": pk["hbm_gbs"],
+                      "peak_source": pk["source"], "l2": "flushed before every launch",
+                      "rows": rows}), flush=True)
+    opt.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -581,13 +626,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
-    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b"])
+    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "sweep":
+        run_sweep(args)
     elif args.workload != "headline":
         args.steps = min(args.steps, 3)
         run_stack(args)
