@@ -50,6 +50,9 @@
 namespace adama {
 namespace {
 
+#ifndef ADAMA_WGRAD_STAGES
+#define ADAMA_WGRAD_STAGES 6  // shared-memory ring depth of the CTA-pair kernel (build-time tunable)
+#endif
 constexpr int BN = 256;     // tile columns (d_out direction) = UMMA N
 constexpr int BK = 64;      // tokens per pipeline stage
 constexpr int UMMA_K = 16;  // tokens per tcgen05.mma (bf16)
@@ -78,7 +81,7 @@ struct Geo {
     static constexpr int A_STAGE_BYTES = A_BOXES * BOX_BYTES;
     static constexpr int B_STAGE_BYTES = B_BOXES * BOX_BYTES;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KB or 32 KB
-    static constexpr int STAGES = CTAS == 1 ? 4 : 6;
+    static constexpr int STAGES = CTAS == 1 ? 4 : ADAMA_WGRAD_STAGES;
     static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
     static constexpr int SMEM_BYTES = SMEM_BAR_OFF + SMEM_BAR_BYTES + 1024;  // + alignment slack
