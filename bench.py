@@ -2,7 +2,7 @@
 """Benchmark of the AdamA hot path on B200: fold / apply GB/s and fused wgrad+fold TFLOP/s.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload headline|gpt2xl|llama7b|sweep]
+                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors]
 
 One step of the headline workload = one pass of the whole path:
   phase A  (flat 335M-parameter buffer, bf16 gradients, N=8):
@@ -619,6 +619,59 @@ def run_sweep(args):
     opt.close()
 
 
+def run_small_tensors(args):
+    """The non-matrix parameters of a GPT-2-XL-shaped model (per block: two norms, four biases;
+    432 tensors, 1.0 M elements): one mini-batch of N=8 folds + apply with the multi-tensor
+    calls against one call per tensor.  GPU time by CUDA events, host time by perf_counter."""
+    import paper_2305_19982_b200 as adama
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    sizes = []
+    for _ in range(wl.CONFIG4_BLOCKS):
+        sizes += [1600, 1600, 4800, 1600, 1600, 1600, 6400, 1600]
+    sizes += [1600, 1600]
+    N = wl.CONFIG4_N_MICRO
+    ws = [wl.normal((n,), 0.02, torch.float32, 10 + i, device=dev) for i, n in enumerate(sizes)]
+    ms = [torch.zeros(n, device=dev) for n in sizes]
+    vs = [torch.zeros(n, device=dev) for n in sizes]
+    gs = [wl.normal((n,), 1e-3, torch.bfloat16, 5000 + i, device=dev) for i, n in enumerate(sizes)]
+    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
+    res = {}
+    for mode in ("multi", "per_tensor"):
+        def step():
+            opt.begin_minibatch(N)
+            for _ in range(N):
+                if mode == "multi":
+                    opt.fold_multi(gs, ms, vs)
+                else:
+                    for g, m, v in zip(gs, ms, vs):
+                        opt.fold(g, m, v)
+            if mode == "multi":
+                opt.apply_multi(ws, ms, vs, wl.LR)
+            else:
+                for w, m, v in zip(ws, ms, vs):
+                    opt.apply(w, m, v, wl.LR)
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        l0 = opt.launch_count
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        host = (time.perf_counter() - t0) / args.steps
+        torch.cuda.synchronize()
+        res[mode] = {"gpu_ms_per_minibatch": e0.elapsed_time(e1) / args.steps,
+                     "host_ms_per_minibatch": host * 1e3,
+                     "launches_per_minibatch": (opt.launch_count - l0) // args.steps}
+    print(json.dumps({"metric": "adama_small_tensor_minibatch_ms", "unit": "ms", "tensors": len(sizes),
+                      "elements": sum(sizes), "n_micro": N, **res}), flush=True)
+    opt.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -626,7 +679,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
-    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep"])
+    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -635,6 +688,9 @@ def main():
         run_reference(args)
     elif args.workload == "sweep":
         run_sweep(args)
+    elif args.workload == "small_tensors":
+        args.steps = min(args.steps, 10)
+        run_small_tensors(args)
     elif args.workload != "headline":
         args.steps = min(args.steps, 3)
         run_stack(args)

@@ -153,6 +153,24 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
 ADAMA_API adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                    double lr, void *cuda_stream);
 
+/* adama_fold for a list of tensors in as few launches as possible (Algorithm 2's inner loop
+ * visits "each layer"; a transformer has hundreds of small ones: biases, norm scales).
+ * grads, m, v, n are HOST arrays of `count` entries: device pointers and element counts; all
+ * gradients share the dtype gdt.  Tensors shorter than 4 Mi elements are grouped, up to 64
+ * per launch, the table travelling in the kernel's parameters (nothing is allocated); longer
+ * ones get the single-tensor kernel.  Same arithmetic and the same per-tensor rules as
+ * adama_fold; results are bit-identical to `count` adama_fold calls.  The arrays are read
+ * before the call returns.  Errors: as adama_fold, for the first offending tensor. */
+ADAMA_API adama_status adama_fold_multi(adama_ctx *ctx, const void *const *grads, adama_dtype gdt,
+                                        float *const *m, float *const *v, const size_t *n,
+                                        int count, void *cuda_stream);
+
+/* adama_apply for a list of tensors, grouped like adama_fold_multi; bit-identical to `count`
+ * adama_apply calls with the same lr. */
+ADAMA_API adama_status adama_apply_multi(adama_ctx *ctx, float *const *w, float *const *m,
+                                         float *const *v, const size_t *n, int count, double lr,
+                                         void *cuda_stream);
+
 /* Data-parallel variant of adama_apply (Section 3.3, Eqs. 4-7): R = world_size devices
  * each fold their own N micro-batches into their own m and v; once per mini-batch the
  * CALLER sums m and v over the devices (one all-reduce each, e.g. NCCL, on the same

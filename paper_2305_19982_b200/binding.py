@@ -17,7 +17,8 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_host", "adama_linear_wgrad_fold_host",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_multi", "adama_apply_multi",
+    "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
     "adama_host_constants_allreduced", "adama_host_constants_sharded",
@@ -79,6 +80,10 @@ def load_library() -> ctypes.CDLL:
                                                   ctypes.POINTER(ctypes.c_float)]
     L.adama_apply_sharded.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
     L.adama_host_constants_sharded.argtypes = L.adama_host_constants_allreduced.argtypes
+    L.adama_fold_multi.argtypes = [vp, ctypes.POINTER(vp), ci, ctypes.POINTER(vp),
+                                   ctypes.POINTER(vp), ctypes.POINTER(sz), ci, vp]
+    L.adama_apply_multi.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                    ctypes.POINTER(sz), ci, dbl, vp]
     L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
     L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
     L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
@@ -215,6 +220,47 @@ class AdamA:
                                         _dev_ptr(m, torch.float32, "m"),
                                         _dev_ptr(v, torch.float32, "v"), n, float(lr),
                                         _stream_ptr(self.device)))
+
+    @staticmethod
+    def _ptr_array(tensors, dtype, name):
+        arr = (ctypes.c_void_p * len(tensors))()
+        for i, t in enumerate(tensors):
+            if not t.is_contiguous():
+                raise ValueError(f"{name}[{i}] must be contiguous")
+            arr[i] = _dev_ptr(t, dtype, f"{name}[{i}]")
+        return arr
+
+    def fold_multi(self, grads, ms, vs) -> None:
+        """adama_fold_multi over lists of tensors (all gradients of one dtype)."""
+        if not (len(grads) == len(ms) == len(vs)):
+            raise ValueError("lists must have equal length")
+        if not grads:
+            return
+        gdtype = grads[0].dtype
+        gdt = {torch.float32: F32, torch.bfloat16: BF16}[gdtype]
+        for g, m, v in zip(grads, ms, vs):
+            if g.numel() != m.numel() or g.numel() != v.numel():
+                raise ValueError("grad, m, v must have the same number of elements")
+        ns = (ctypes.c_size_t * len(grads))(*[g.numel() for g in grads])
+        self._check(self._L.adama_fold_multi(
+            self._h, self._ptr_array(grads, gdtype, "grads"), gdt,
+            self._ptr_array(ms, torch.float32, "m"), self._ptr_array(vs, torch.float32, "v"), ns,
+            len(grads), _stream_ptr(self.device)))
+
+    def apply_multi(self, ws, ms, vs, lr: float) -> None:
+        """adama_apply_multi over lists of tensors."""
+        if not (len(ws) == len(ms) == len(vs)):
+            raise ValueError("lists must have equal length")
+        if not ws:
+            return
+        for w, m, v in zip(ws, ms, vs):
+            if w.numel() != m.numel() or w.numel() != v.numel():
+                raise ValueError("w, m, v must have the same number of elements")
+        ns = (ctypes.c_size_t * len(ws))(*[w.numel() for w in ws])
+        self._check(self._L.adama_apply_multi(
+            self._h, self._ptr_array(ws, torch.float32, "w"), self._ptr_array(ms, torch.float32, "m"),
+            self._ptr_array(vs, torch.float32, "v"), ns, len(ws), float(lr),
+            _stream_ptr(self.device)))
 
     def apply_allreduced(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float,
                          world_size: int) -> None:

@@ -276,6 +276,93 @@ adama_status adama_apply_sharded(adama_ctx *ctx, float *w, float *m, float *v, s
     return apply_impl(ctx, w, m, v, n, lr, world_size, true, cuda_stream);
 }
 
+// ---- multi-tensor forms ---------------------------------------------------------------------
+
+// Tensors at least this long go to the single-tensor kernels (they saturate the GPU alone).
+static const size_t kMultiLargeThreshold = (size_t)1 << 22;
+
+adama_status adama_fold_multi(adama_ctx *ctx, const void *const *grads, adama_dtype gdt,
+                              float *const *m, float *const *v, const size_t *n, int count,
+                              void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (count < 0 || (count > 0 && (!grads || !m || !v || !n)))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "fold_multi: null list or negative count");
+    for (int i = 0; i < count; ++i) {
+        adama_status st = check_fold_args(ctx, grads[i], gdt, m[i], v[i], n[i]);
+        if (st != ADAMA_OK) return st;
+    }
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const void *g_[adama::kMultiMax];
+    float *m_[adama::kMultiMax], *v_[adama::kMultiMax];
+    size_t n_[adama::kMultiMax];
+    int k = 0;
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i <= count && e == cudaSuccess; ++i) {
+        const bool flush = (i == count) || k == adama::kMultiMax;
+        if (flush && k > 0) {
+            e = adama::launch_fold_multi(g_, gdt, m_, v_, n_, k, ctx->fold_c, ctx->sm_count, stream);
+            ctx->launches += 1;
+            k = 0;
+        }
+        if (i == count || e != cudaSuccess) break;
+        if (n[i] == 0) continue;
+        if (n[i] >= kMultiLargeThreshold) {
+            e = adama::launch_fold(grads[i], gdt, m[i], v[i], n[i], ctx->fold_c, ctx->sm_count, stream);
+            ctx->launches += 1;
+            continue;
+        }
+        g_[k] = grads[i];
+        m_[k] = m[i];
+        v_[k] = v[i];
+        n_[k] = n[i];
+        ++k;
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, "fold_multi launch", e);
+    return ADAMA_OK;
+}
+
+adama_status adama_apply_multi(adama_ctx *ctx, float *const *w, float *const *m, float *const *v,
+                               const size_t *n, int count, double lr, void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (count < 0 || (count > 0 && (!w || !m || !v || !n)))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply_multi: null list or negative count");
+    for (int i = 0; i < count; ++i) {
+        adama_status st = check_apply_args(ctx, w[i], m[i], v[i], n[i], lr);
+        if (st != ADAMA_OK) return st;
+    }
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const adama::ApplyConstants c =
+        adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr);
+    float *w_[adama::kMultiMax], *m_[adama::kMultiMax], *v_[adama::kMultiMax];
+    size_t n_[adama::kMultiMax];
+    int k = 0;
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i <= count && e == cudaSuccess; ++i) {
+        const bool flush = (i == count) || k == adama::kMultiMax;
+        if (flush && k > 0) {
+            e = adama::launch_apply_multi(w_, m_, v_, n_, k, c, ctx->sm_count, stream);
+            ctx->launches += 1;
+            k = 0;
+        }
+        if (i == count || e != cudaSuccess) break;
+        if (n[i] == 0) continue;
+        if (n[i] >= kMultiLargeThreshold) {
+            e = adama::launch_apply(w[i], m[i], v[i], n[i], c, ctx->sm_count, stream);
+            ctx->launches += 1;
+            continue;
+        }
+        w_[k] = w[i];
+        m_[k] = m[i];
+        v_[k] = v[i];
+        n_[k] = n[i];
+        ++k;
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, "apply_multi launch", e);
+    return ADAMA_OK;
+}
+
 // ---- host-buffer variants -------------------------------------------------------------------
 
 adama_status adama_fold_host(adama_ctx *ctx, const void *grad_host, adama_dtype gdt, float *m,

@@ -47,6 +47,15 @@ cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, s
 cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants c, int sm_count,
                          cudaStream_t stream);
 
+// multi-tensor forms (multi_tensor.cu): up to kMultiMax tensors per launch, each shorter than
+// 2^32 * 4096 elements in total blocks
+constexpr int kMultiMax = 64;
+cudaError_t launch_fold_multi(const void *const *g, adama_dtype gdt, float *const *m,
+                              float *const *v, const size_t *n, int count, FoldConstants c,
+                              int sm_count, cudaStream_t stream);
+cudaError_t launch_apply_multi(float *const *w, float *const *m, float *const *v, const size_t *n,
+                               int count, ApplyConstants c, int sm_count, cudaStream_t stream);
+
 // fused weight-gradient + fold (wgrad_fold.cu)
 struct WgradArgs {
     const void *X;
