@@ -636,18 +636,19 @@ def run_small_tensors(args):
     vs = [torch.zeros(n, device=dev) for n in sizes]
     gs = [wl.normal((n,), 1e-3, torch.bfloat16, 5000 + i, device=dev) for i, n in enumerate(sizes)]
     opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
+    gl, ml, vl, wlst = (adama.TensorList(x) for x in (gs, ms, vs, ws))  # marshalled once
     res = {}
     for mode in ("multi", "per_tensor"):
         def step():
             opt.begin_minibatch(N)
             for _ in range(N):
                 if mode == "multi":
-                    opt.fold_multi(gs, ms, vs)
+                    opt.fold_multi(gl, ml, vl)
                 else:
                     for g, m, v in zip(gs, ms, vs):
                         opt.fold(g, m, v)
             if mode == "multi":
-                opt.apply_multi(ws, ms, vs, wl.LR)
+                opt.apply_multi(wlst, ml, vl, wl.LR)
             else:
                 for w, m, v in zip(ws, ms, vs):
                     opt.apply(w, m, v, wl.LR)

@@ -6,8 +6,8 @@ module only marshals arguments (device pointers of torch tensors, the current
 stream).  There is no CPU fallback: importing works without a GPU, but creating
 an ``AdamA`` context raises if the library or a sm_100 device is missing.
 """
-from .binding import (AdamA, AdamAError, Status, library_path, load_library, host_constants,
+from .binding import (AdamA, AdamAError, TensorList, Status, library_path, load_library, host_constants,
                       linear_wgrad_fold_noalloc, EXPORTED_SYMBOLS)
 
-__all__ = ["AdamA", "AdamAError", "Status", "library_path", "load_library", "host_constants",
+__all__ = ["AdamA", "AdamAError", "TensorList", "Status", "library_path", "load_library", "host_constants",
            "linear_wgrad_fold_noalloc", "EXPORTED_SYMBOLS"]

@@ -130,6 +130,25 @@ def _dev_ptr(t: torch.Tensor, dtype: torch.dtype, name: str) -> int:
     return t.data_ptr()
 
 
+class TensorList:
+    """Device pointers and sizes of a list of contiguous CUDA tensors, marshalled once for
+    repeated multi-tensor calls (keeps the tensors alive)."""
+
+    def __init__(self, tensors, dtype=None):
+        self.tensors = list(tensors)
+        self.dtype = dtype if dtype is not None else (self.tensors[0].dtype if self.tensors else torch.float32)
+        self.ptrs = (ctypes.c_void_p * len(self.tensors))()
+        for i, t in enumerate(self.tensors):
+            if not t.is_contiguous():
+                raise ValueError(f"tensor {i} must be contiguous")
+            self.ptrs[i] = _dev_ptr(t, self.dtype, f"tensor {i}")
+        self.numels = [t.numel() for t in self.tensors]
+        self.ns = (ctypes.c_size_t * len(self.tensors))(*self.numels)
+
+    def __len__(self):
+        return len(self.tensors)
+
+
 class AdamA:
     """One AdamA context (adama_ctx) bound to a CUDA device.
 
@@ -221,46 +240,35 @@ class AdamA:
                                         _dev_ptr(v, torch.float32, "v"), n, float(lr),
                                         _stream_ptr(self.device)))
 
-    @staticmethod
-    def _ptr_array(tensors, dtype, name):
-        arr = (ctypes.c_void_p * len(tensors))()
-        for i, t in enumerate(tensors):
-            if not t.is_contiguous():
-                raise ValueError(f"{name}[{i}] must be contiguous")
-            arr[i] = _dev_ptr(t, dtype, f"{name}[{i}]")
-        return arr
-
     def fold_multi(self, grads, ms, vs) -> None:
-        """adama_fold_multi over lists of tensors (all gradients of one dtype)."""
+        """adama_fold_multi over lists of tensors (all gradients of one dtype); pass TensorList
+        objects to skip the per-call marshalling."""
+        grads = grads if isinstance(grads, TensorList) else TensorList(grads)
+        ms = ms if isinstance(ms, TensorList) else TensorList(ms, torch.float32)
+        vs = vs if isinstance(vs, TensorList) else TensorList(vs, torch.float32)
         if not (len(grads) == len(ms) == len(vs)):
             raise ValueError("lists must have equal length")
-        if not grads:
+        if len(grads) == 0:
             return
-        gdtype = grads[0].dtype
-        gdt = {torch.float32: F32, torch.bfloat16: BF16}[gdtype]
-        for g, m, v in zip(grads, ms, vs):
-            if g.numel() != m.numel() or g.numel() != v.numel():
-                raise ValueError("grad, m, v must have the same number of elements")
-        ns = (ctypes.c_size_t * len(grads))(*[g.numel() for g in grads])
-        self._check(self._L.adama_fold_multi(
-            self._h, self._ptr_array(grads, gdtype, "grads"), gdt,
-            self._ptr_array(ms, torch.float32, "m"), self._ptr_array(vs, torch.float32, "v"), ns,
-            len(grads), _stream_ptr(self.device)))
+        if grads.numels != ms.numels or grads.numels != vs.numels:
+            raise ValueError("grad, m, v must have the same number of elements")
+        gdt = {torch.float32: F32, torch.bfloat16: BF16}[grads.dtype]
+        self._check(self._L.adama_fold_multi(self._h, grads.ptrs, gdt, ms.ptrs, vs.ptrs, grads.ns,
+                                             len(grads), _stream_ptr(self.device)))
 
     def apply_multi(self, ws, ms, vs, lr: float) -> None:
-        """adama_apply_multi over lists of tensors."""
+        """adama_apply_multi over lists of tensors (or TensorList objects)."""
+        ws = ws if isinstance(ws, TensorList) else TensorList(ws, torch.float32)
+        ms = ms if isinstance(ms, TensorList) else TensorList(ms, torch.float32)
+        vs = vs if isinstance(vs, TensorList) else TensorList(vs, torch.float32)
         if not (len(ws) == len(ms) == len(vs)):
             raise ValueError("lists must have equal length")
-        if not ws:
+        if len(ws) == 0:
             return
-        for w, m, v in zip(ws, ms, vs):
-            if w.numel() != m.numel() or w.numel() != v.numel():
-                raise ValueError("w, m, v must have the same number of elements")
-        ns = (ctypes.c_size_t * len(ws))(*[w.numel() for w in ws])
-        self._check(self._L.adama_apply_multi(
-            self._h, self._ptr_array(ws, torch.float32, "w"), self._ptr_array(ms, torch.float32, "m"),
-            self._ptr_array(vs, torch.float32, "v"), ns, len(ws), float(lr),
-            _stream_ptr(self.device)))
+        if ws.numels != ms.numels or ws.numels != vs.numels:
+            raise ValueError("w, m, v must have the same number of elements")
+        self._check(self._L.adama_apply_multi(self._h, ws.ptrs, ms.ptrs, vs.ptrs, ws.ns, len(ws),
+                                              float(lr), _stream_ptr(self.device)))
 
     def apply_allreduced(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float,
                          world_size: int) -> None:
