@@ -153,6 +153,16 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
 ADAMA_API adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                    double lr, void *cuda_stream);
 
+/* The bias of the same linear layer: its raw micro-batch gradient is the column sum of dY,
+ *     g[q] = sum_{tau < tokens} dY[tau,q],   m[q] += a*g[q],   v[q] += b*g[q]^2
+ * (Algorithm 2, inner loop body; the sum over tokens is completed on-chip, by a cluster of
+ * CTAs through distributed shared memory, before it is squared).  dY as in
+ * adama_linear_wgrad_fold (bf16, row pitch ldy, 16-byte aligned, ldy a multiple of 8);
+ * m, v: d_out fp32 elements each, contiguous.  tokens == 0 is a no-op.  Deterministic.
+ * Errors: INVALID_ARG, BAD_STATE, MISALIGNED, CUDA. */
+ADAMA_API adama_status adama_bias_grad_fold(adama_ctx *ctx, const void *dY, int tokens, int d_out,
+                                            int64_t ldy, float *m, float *v, void *cuda_stream);
+
 /* adama_fold for a list of tensors in as few launches as possible (Algorithm 2's inner loop
  * visits "each layer"; a transformer has hundreds of small ones: biases, norm scales).
  * grads, m, v, n are HOST arrays of `count` entries: device pointers and element counts; all

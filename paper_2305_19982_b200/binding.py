@@ -17,7 +17,7 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_multi", "adama_apply_multi",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
@@ -84,6 +84,7 @@ def load_library() -> ctypes.CDLL:
                                    ctypes.POINTER(vp), ctypes.POINTER(sz), ci, vp]
     L.adama_apply_multi.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
                                     ctypes.POINTER(sz), ci, dbl, vp]
+    L.adama_bias_grad_fold.argtypes = [vp, vp, ci, ci, i64, vp, vp, vp]
     L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
     L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
     L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
@@ -239,6 +240,19 @@ class AdamA:
                                         _dev_ptr(m, torch.float32, "m"),
                                         _dev_ptr(v, torch.float32, "v"), n, float(lr),
                                         _stream_ptr(self.device)))
+
+    def bias_grad_fold(self, dY: torch.Tensor, m: torch.Tensor, v: torch.Tensor) -> None:
+        """adama_bias_grad_fold: dY [tokens, d_out] bf16 (unit stride in the last dim), m, v [d_out]."""
+        tokens, d_out = dY.shape
+        if dY.shape[1] > 1 and dY.stride(1) != 1:
+            raise ValueError("dY must have unit stride in its last dimension")
+        if m.numel() != d_out or v.numel() != d_out or not (m.is_contiguous() and v.is_contiguous()):
+            raise ValueError("m, v must be contiguous with d_out elements")
+        ldy = dY.stride(0) if tokens > 1 else max(d_out, dY.stride(0))
+        self._check(self._L.adama_bias_grad_fold(
+            self._h, _dev_ptr(dY, torch.bfloat16, "dY"), tokens, d_out, ldy,
+            _dev_ptr(m, torch.float32, "m"), _dev_ptr(v, torch.float32, "v"),
+            _stream_ptr(self.device)))
 
     def fold_multi(self, grads, ms, vs) -> None:
         """adama_fold_multi over lists of tensors (all gradients of one dtype); pass TensorList

@@ -276,6 +276,25 @@ adama_status adama_apply_sharded(adama_ctx *ctx, float *w, float *m, float *v, s
     return apply_impl(ctx, w, m, v, n, lr, world_size, true, cuda_stream);
 }
 
+adama_status adama_bias_grad_fold(adama_ctx *ctx, const void *dY, int tokens, int d_out,
+                                  int64_t ldy, float *m, float *v, void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (tokens < 0 || d_out < 1 || !m || !v || (tokens > 0 && !dY) || ldy < d_out)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "bias_grad_fold: bad shape, null pointer or pitch");
+    if (ctx->n_micro < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "bias_grad_fold: adama_begin_minibatch has not been called");
+    if (!aligned_to(dY, 16) || ldy % 8 || !aligned_to(m, 4) || !aligned_to(v, 4))
+        return fail(ctx, ADAMA_ERR_MISALIGNED,
+                    "bias_grad_fold: dY must be 16-byte aligned with ldy a multiple of 8");
+    if (tokens == 0) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaError_t e = adama::launch_bias_grad_fold(dY, tokens, d_out, ldy, m, v, ctx->fold_c,
+                                                 static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "bias_grad_fold launch", e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
 // ---- multi-tensor forms ---------------------------------------------------------------------
 
 // Tensors at least this long go to the single-tensor kernels (they saturate the GPU alone).
