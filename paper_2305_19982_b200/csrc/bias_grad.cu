@@ -3,7 +3,7 @@
 //     m[q] += a*g[q];  v[q] += b*g[q]^2              (Algorithm 2, inner loop body)
 // The token sum must be complete before it is squared, so the partial sums of the CTAs that
 // share a column slab are combined on-chip: a cluster of 8 CTAs splits the tokens, each leaves
-// its 128 partial sums in shared memory, and the cluster's first CTA adds the eight vectors
+// its 256 partial sums in shared memory, and the cluster's first CTA adds the eight vectors
 // through distributed shared memory, in rank order (deterministic), and folds.  One pass over
 // dY (2*tokens*d_out bytes), nothing written but m and v.
 #include <cooperative_groups.h>
@@ -16,8 +16,10 @@ namespace cg = cooperative_groups;
 namespace adama {
 namespace {
 
-constexpr int kSlabCols = 128;  // columns per cluster: 32 threads x 4 bf16 (8 bytes each)
-constexpr int kRowLanes = 8;    // rows read concurrently by one CTA
+constexpr int kColsPerThread = 8;                  // 8 bf16 = one 16-byte load
+constexpr int kSlabCols = 32 * kColsPerThread;     // 256 columns per cluster
+constexpr int kRowLanes = 16;                      // rows read concurrently by one CTA
+constexpr int kUnroll = 8;                         // independent 16-byte loads in flight per thread
 constexpr int kThreads = 32 * kRowLanes;
 constexpr int kClusterSize = 8;  // CTAs that split the tokens of one slab
 
@@ -28,30 +30,50 @@ bias_grad_fold_kernel(const __nv_bfloat16 *__restrict__ dY, int tokens, int d_ou
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned rank = cluster.block_rank();
     const int slab = blockIdx.x / kClusterSize;
-    const int cgp = threadIdx.x & 31;  // column group: 4 columns
+    const int cgp = threadIdx.x & 31;  // column group: 8 columns
     const int rl = threadIdx.x >> 5;   // row lane
-    const int col = slab * kSlabCols + cgp * 4;
+    const int col = slab * kSlabCols + cgp * kColsPerThread;
     // this CTA's share of the tokens
     const int per = (tokens + kClusterSize - 1) / kClusterSize;
     const int t0 = (int)rank * per;
     const int t1 = t0 + per < tokens ? t0 + per : tokens;
 
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    if (col + 3 < d_out) {
-        for (int tau = t0 + rl; tau < t1; tau += kRowLanes) {
-            const uint2 x = *reinterpret_cast<const uint2 *>(dY + (long long)tau * ldy + col);
-            acc[0] += __uint_as_float(x.x << 16);
-            acc[1] += __uint_as_float(x.x & 0xffff0000u);
-            acc[2] += __uint_as_float(x.y << 16);
-            acc[3] += __uint_as_float(x.y & 0xffff0000u);
+    float acc[kColsPerThread];
+#pragma unroll
+    for (int e = 0; e < kColsPerThread; ++e) acc[e] = 0.f;
+    if (col + kColsPerThread <= d_out) {
+        int tau = t0 + rl;
+        for (; tau + (kUnroll - 1) * kRowLanes < t1; tau += kUnroll * kRowLanes) {
+            uint4 x[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                x[u] = *reinterpret_cast<const uint4 *>(dY + (long long)(tau + u * kRowLanes) * ldy + col);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const unsigned wds[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    acc[2 * k] += __uint_as_float(wds[k] << 16);
+                    acc[2 * k + 1] += __uint_as_float(wds[k] & 0xffff0000u);
+                }
+            }
+        }
+        for (; tau < t1; tau += kRowLanes) {
+            const uint4 x = *reinterpret_cast<const uint4 *>(dY + (long long)tau * ldy + col);
+            const unsigned wds[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[2 * k] += __uint_as_float(wds[k] << 16);
+                acc[2 * k + 1] += __uint_as_float(wds[k] & 0xffff0000u);
+            }
         }
     } else {
         for (int tau = t0 + rl; tau < t1; tau += kRowLanes)
-            for (int e = 0; e < 4; ++e)
+            for (int e = 0; e < kColsPerThread; ++e)
                 if (col + e < d_out) acc[e] += __bfloat162float(dY[(long long)tau * ldy + col + e]);
     }
 #pragma unroll
-    for (int e = 0; e < 4; ++e) part[rl][cgp * 4 + e] = acc[e];
+    for (int e = 0; e < kColsPerThread; ++e) part[rl][cgp * kColsPerThread + e] = acc[e];
     __syncthreads();
     // row lanes -> one vector per CTA, kept in part[0]
     if (threadIdx.x < kSlabCols) {
