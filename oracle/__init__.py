@@ -53,6 +53,11 @@ def load(path) -> ctypes.CDLL:
     L.oracle_update.argtypes = [_c_double_p, _c_double_p, _c_double_p, ctypes.c_size_t,
                                 ctypes.c_long, ctypes.c_double, ctypes.c_double,
                                 ctypes.c_double, ctypes.c_double]
+    L.oracle_update_decoupled_decay.argtypes = [_c_double_p, _c_double_p, _c_double_p,
+                                                ctypes.c_size_t, ctypes.c_long, ctypes.c_double,
+                                                ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                                ctypes.c_double]
+    L.oracle_update_decoupled_decay.restype = None
     L.oracle_closed_form_moments.argtypes = [_c_double_p, _c_double_p, _c_double_p,
                                              ctypes.c_size_t, ctypes.c_int, ctypes.c_double,
                                              ctypes.c_double, ctypes.c_int]
@@ -176,11 +181,17 @@ class AdamAOracle:
         [d_in, d_out] weights live at [lo, lo + d_in*d_out)."""
         self.fold(linear_wgrad(X, dY), lo)
 
-    def update(self, lr: float) -> None:
-        """Bias-corrected Adam step with the current t."""
+    def update(self, lr: float, weight_decay: float = 0.0) -> None:
+        """Bias-corrected Adam step with the current t; weight_decay > 0 adds AdamW's
+        decoupled decay (an extension, not part of the paper's algorithms)."""
         assert self.t >= 1
-        lib().oracle_update(_p(self.theta), _p(self.m), _p(self.v), self.n, self.t, float(lr),
-                            self.beta1, self.beta2, self.eps)
+        if weight_decay == 0.0:
+            lib().oracle_update(_p(self.theta), _p(self.m), _p(self.v), self.n, self.t, float(lr),
+                                self.beta1, self.beta2, self.eps)
+        else:
+            lib().oracle_update_decoupled_decay(_p(self.theta), _p(self.m), _p(self.v), self.n,
+                                                self.t, float(lr), self.beta1, self.beta2,
+                                                self.eps, float(weight_decay))
 
 
 class AdamADDPOracle:

@@ -86,6 +86,24 @@ ORACLE_API void oracle_update(double *theta, const double *m, const double *v, s
     }
 }
 
+/* Extension outside the paper's algorithms (its Discussion only remarks that other
+ * momentum optimizers can take the same accumulation): the update above with decoupled
+ * weight decay as in AdamW (Loshchilov & Hutter, "Decoupled Weight Decay Regularization",
+ * Algorithm 2):  theta <- theta - alpha*lambda*theta - alpha*m_hat/(sqrt(v_hat)+eps).
+ * lambda = 0 is oracle_update. */
+ORACLE_API void oracle_update_decoupled_decay(double *theta, const double *m, const double *v,
+                                              size_t n, long t, double alpha, double beta1,
+                                              double beta2, double eps, double lambda) {
+    double c1 = 1.0 - pow(beta1, (double)t);
+    double c2 = 1.0 - pow(beta2, (double)t);
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t k = 0; k < (ptrdiff_t)n; ++k) {
+        double m_hat = m[k] / c1;
+        double v_hat = v[k] / c2;
+        theta[k] = theta[k] - alpha * lambda * theta[k] - alpha * m_hat / (sqrt(v_hat) + eps);
+    }
+}
+
 /* Algorithm 1, the two moment lines, evaluated per mini-batch from the stored
  * list of raw micro-batch gradients grads[i*n + k], i < N:
  *     g_i = grads_i / N

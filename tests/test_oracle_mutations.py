@@ -23,6 +23,9 @@ MUTATIONS = {
     "ddp v not pre-scaled": ("v[k] = (double)devices * beta2 * v[k];", "v[k] = beta2 * v[k];"),
     "closed form: adam/adama swapped": ("adam_variant ? sum_g * sum_g : sum_g2",
                                         "adam_variant ? sum_g2 : sum_g * sum_g"),
+    "weight decay coupled into the gradient term": (
+        "theta[k] - alpha * lambda * theta[k] - alpha * m_hat / (sqrt(v_hat) + eps)",
+        "theta[k] - alpha * (m_hat + lambda * theta[k]) / (sqrt(v_hat) + eps)"),
     "wgrad accumulates |x|": ("acc += X[(size_t)tau * ldx + (size_t)p] * dY",
                               "acc += fabs(X[(size_t)tau * ldx + (size_t)p]) * dY"),
 }
@@ -33,6 +36,7 @@ def _run_all_pins():
     pins.test_worked_example_adam_variant_differs()
     for eps in (1e-8, 1e-3):
         pins.test_n1_is_standard_adam(eps)
+    pins.test_n1_with_decoupled_decay_is_torch_adamw()
     pins.test_first_moment_is_adams_on_mean_gradient(4)
     pins.test_identical_micro_gradients_give_adam_v_over_n(3)
     pins.test_cauchy_schwarz_bound_and_sign()

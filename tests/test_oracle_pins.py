@@ -102,6 +102,30 @@ def test_n1_is_standard_adam(eps):
         np.testing.assert_allclose(orc.theta, p.detach().numpy(), rtol=1e-13, atol=0)
 
 
+def test_n1_with_decoupled_decay_is_torch_adamw():
+    """The weight-decay extension: N=1 equals torch.optim.AdamW (fp64) step by step."""
+    rng = np.random.default_rng(31)
+    n, wd = 40, 0.05
+    theta0 = rng.normal(0, 0.5, n)
+    orc = AdamAOracle(theta0, B1, B2, EPS)
+    p = torch.nn.Parameter(torch.tensor(theta0, dtype=torch.float64))
+    opt = torch.optim.AdamW([p], lr=LR, betas=(B1, B2), eps=EPS, weight_decay=wd, amsgrad=False,
+                            foreach=False, fused=False)
+    for step in range(5):
+        g = rng.normal(0, 1e-2, n)
+        orc.begin_minibatch(1)
+        orc.fold(g)
+        orc.update(LR, weight_decay=wd)
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(orc.theta, p.detach().numpy(), rtol=1e-13, atol=0)
+    plain = AdamAOracle(theta0, B1, B2, EPS)
+    plain.begin_minibatch(1)
+    plain.fold(g)
+    plain.update(LR)
+    assert not np.allclose(plain.theta, theta0 * (1 - LR * wd), rtol=1e-9)
+
+
 @pytest.mark.parametrize("N", [2, 4, 8])
 def test_first_moment_is_adams_on_mean_gradient(N):
     rng = np.random.default_rng(5 + N)
