@@ -286,6 +286,14 @@ ADAMA_API adama_status adama_set_step(adama_ctx *ctx, int64_t t);
 /* Micro-batch count fixed by the last begin_minibatch (0 before the first). */
 ADAMA_API int adama_get_n_micro(const adama_ctx *ctx);
 
+/* Extension beyond the paper's algorithms (its Discussion notes that other momentum-based
+ * optimizers can use the same accumulation): decoupled weight decay as in AdamW.  With
+ * weight_decay = lambda > 0 every later apply computes
+ *     w <- w*(1 - lr*lambda) - lr * m_hat / (sqrt(v_hat) + eps)
+ * (the decay is not folded into m or v).  lambda = 0, the default, is Algorithm 2 exactly
+ * (the factor is 1.0f, results are bit-identical).  Errors: INVALID_ARG (negative or not finite). */
+ADAMA_API adama_status adama_set_weight_decay(adama_ctx *ctx, double weight_decay);
+
 /* Waits for `cuda_stream`, then reads and clears the device status block.
  * Returns ADAMA_OK, ADAMA_ERR_TIMEOUT (a bounded wait inside the fused kernel
  * expired; m and v of that call are incomplete) or ADAMA_ERR_CUDA. */

@@ -19,7 +19,7 @@ EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
     "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
-    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro",
+    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
     "adama_host_constants_allreduced", "adama_host_constants_sharded",
     "adama_version",
@@ -94,6 +94,7 @@ def load_library() -> ctypes.CDLL:
     L.adama_get_step.restype = i64
     L.adama_set_step.argtypes = [vp, i64]
     L.adama_get_n_micro.argtypes = [vp]
+    L.adama_set_weight_decay.argtypes = [vp, dbl]
     L.adama_sync_status.argtypes = [vp, vp]
     L.adama_last_error.argtypes = [vp]
     L.adama_last_error.restype = ctypes.c_char_p
@@ -360,6 +361,10 @@ class AdamA:
 
     def set_step(self, t: int) -> None:
         self._check(self._L.adama_set_step(self._h, int(t)))
+
+    def set_weight_decay(self, weight_decay: float) -> None:
+        """adama_set_weight_decay: decoupled (AdamW) decay for all later applies; 0 turns it off."""
+        self._check(self._L.adama_set_weight_decay(self._h, float(weight_decay)))
 
     @property
     def n_micro(self) -> int:

@@ -17,6 +17,7 @@ struct adama_ctx {
     cudaStream_t copy_stream;  // host-buffer variants: H2D copies overlap the folds
     cudaEvent_t ev_copied[2], ev_folded[2], ev_entry;
     int64_t launches;
+    double weight_decay;  // decoupled (AdamW) decay; 0 = the paper's plain update
     char err[256];
 };
 
@@ -36,7 +37,7 @@ static void split_hi_lo(double x, float *hi, float *lo) {
 }
 
 ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr,
-                                    int world, bool sharded) {
+                                    int world, bool sharded, double weight_decay) {
     ApplyConstants c;
     const double R = (double)world;
     double bc1 = 1.0 - pow(beta1, (double)t);
@@ -45,6 +46,7 @@ ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int6
     c.step = (float)(lr / bc1 / R);
     c.inv_bc2 = (float)(1.0 / bc2 / (R * R));
     c.eps = (float)eps;
+    c.w_keep = (float)(1.0 - lr * weight_decay);
     // stored for the next mini-batch: beta1*m_t = (beta1/R)*m and R*beta2*v_t = (beta2/R)*v
     // (sharded: the owner keeps R*beta1*m_t = beta1*m and R^2*beta2*v_t = beta2*v)
     split_hi_lo(sharded ? beta1 : beta1 / R, &c.beta1_hi, &c.beta1_lo);
@@ -253,7 +255,8 @@ static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, siz
     if (n == 0) return ADAMA_OK;
     DeviceGuard guard(ctx->cfg.device);
     adama::ApplyConstants c = adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2,
-                                                          ctx->cfg.eps, ctx->t, lr, world, sharded);
+                                                          ctx->cfg.eps, ctx->t, lr, world, sharded,
+                                                          ctx->weight_decay);
     cudaError_t e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
                                         static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "apply launch", e);
@@ -352,8 +355,8 @@ adama_status adama_apply_multi(adama_ctx *ctx, float *const *w, float *const *m,
     }
     DeviceGuard guard(ctx->cfg.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const adama::ApplyConstants c =
-        adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr);
+    const adama::ApplyConstants c = adama::make_apply_constants(
+        ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr, 1, false, ctx->weight_decay);
     float *w_[adama::kMultiMax], *m_[adama::kMultiMax], *v_[adama::kMultiMax];
     size_t n_[adama::kMultiMax];
     int k = 0;
@@ -483,6 +486,14 @@ adama_status adama_set_step(adama_ctx *ctx, int64_t t) {
 }
 
 int adama_get_n_micro(const adama_ctx *ctx) { return ctx ? ctx->n_micro : -1; }
+
+adama_status adama_set_weight_decay(adama_ctx *ctx, double weight_decay) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (!(weight_decay >= 0.0) || !isfinite(weight_decay))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "set_weight_decay: must be finite and >= 0");
+    ctx->weight_decay = weight_decay;
+    return ADAMA_OK;
+}
 
 adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream) {
     if (!ctx) return ADAMA_ERR_INVALID_ARG;

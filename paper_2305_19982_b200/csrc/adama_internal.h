@@ -25,6 +25,7 @@ struct ApplyConstants {
     float beta1_lo;  // formed as fma(m, hi, m*lo), free of the per-step bias of a
     float beta2_hi;  // plain fp32 beta that would build up over ~1/(1-beta) steps
     float beta2_lo;
+    float w_keep;    // 1 - lr*weight_decay (decoupled decay, AdamW); exactly 1 when it is off
 };
 
 FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsigned flags);
@@ -35,7 +36,7 @@ FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsig
 // states and stay un-normalised between mini-batches (beta*sum instead of beta/R*sum),
 // because the other ranks restart their accumulators for that shard from zero.
 ApplyConstants make_apply_constants(double beta1, double beta2, double eps, int64_t t, double lr,
-                                    int world = 1, bool sharded = false);
+                                    int world = 1, bool sharded = false, double weight_decay = 0.0);
 
 // Status block in device memory (256 bytes): word 0 = first error code recorded
 // by a kernel (0 = none), word 1 = which wait, word 2 = tile; rest reserved.

@@ -150,7 +150,7 @@ fold_scalar_kernel(const G *__restrict__ grad, float *__restrict__ m, float *__r
 // w -= step * m / (sqrt(v*inv_bc2) + eps);  m *= beta1;  v *= beta2
 __device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
     float denom = sqrtf(v * c.inv_bc2) + c.eps;  // IEEE sqrt
-    w = fmaf(-c.step, m / denom, w);             // IEEE division
+    w = fmaf(-c.step, m / denom, w * c.w_keep);             // IEEE division
     // beta = hi + lo: the small product is rounded first (its error is ~1e-15 relative to
     // the result), then one fma rounds x*hi + x*lo once.  The other order would round
     // x*hi first and lose the sub-ulp correction every time.

@@ -93,7 +93,7 @@ fold_multi_kernel(const __grid_constant__ MultiTable tab, float a, float b) {
 
 __device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
     const float denom = sqrtf(v * c.inv_bc2) + c.eps;
-    w = fmaf(-c.step, m / denom, w);
+    w = fmaf(-c.step, m / denom, w * c.w_keep);
     m = fmaf(m, c.beta1_hi, m * c.beta1_lo);
     v = fmaf(v, c.beta2_hi, v * c.beta2_lo);
 }

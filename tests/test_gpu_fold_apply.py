@@ -168,3 +168,39 @@ def test_full_size_config2_sampled():
     assert bool((v >= 0).all()) and bool(torch.isfinite(w).all()) and bool(torch.isfinite(m).all())
     opt.sync_status()
     opt.close()
+
+
+def test_decoupled_weight_decay_extension():
+    """adama_set_weight_decay (AdamW-style, beyond the paper's algorithms) against the oracle's
+    pinned decoupled-decay update; and lambda = 0 stays bit-identical to the plain update."""
+    n, N, wd = 70_001, 2, 0.1
+    w0 = wl.normal((n,), 0.5, torch.float32, 12)
+    orc = AdamAOracle(f64(w0))
+    opt = adama.AdamA()
+    opt.set_weight_decay(wd)
+    plain, zero = adama.AdamA(), adama.AdamA()
+    zero.set_weight_decay(0.0)
+    w, m, v = w0.cuda(), torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    wp, mp, vp = w0.cuda(), torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    wz, mz, vz = w0.cuda(), torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    for step in range(3):
+        for o in (opt, plain, zero):
+            o.begin_minibatch(N)
+        orc.begin_minibatch(N)
+        for i in range(N):
+            g = wl.normal((n,), 1e-2, torch.float32, 300 + 10 * step + i)
+            opt.fold(g.cuda(), m, v)
+            plain.fold(g.cuda(), mp, vp)
+            zero.fold(g.cuda(), mz, vz)
+            orc.fold(f64(g))
+        opt.apply(w, m, v, wl.LR)
+        plain.apply(wp, mp, vp, wl.LR)
+        zero.apply(wz, mz, vz, wl.LR)
+        orc.update(wl.LR, weight_decay=wd)
+        assert rel_l2(f64(w), orc.theta) <= TOL
+        assert torch.equal(wp, wz)
+    assert not torch.equal(w, wp)
+    with pytest.raises(adama.AdamAError):
+        opt.set_weight_decay(-1.0)
+    for o in (opt, plain, zero):
+        o.close()
