@@ -183,6 +183,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
             : "memory");
     }
 }
+// Same, through a 3-D view {64 features, tokens, 64-feature groups}: one operation brings
+// several 64-feature groups (boxes of 8192 bytes, one after the other in shared memory).
+template <int CTAS>
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int tok, int grp,
+                                            uint32_t bar) {
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+            "l"(map), "r"(0), "r"(tok), "r"(grp), "r"(bar)
+            : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+            "l"(map), "r"(0), "r"(tok), "r"(grp), "r"(bar)
+            : "memory");
+    }
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -351,7 +370,11 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
 template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
-                  const __grid_constant__ CUtensorMap map_dy, float *__restrict__ m_out,
+                  const __grid_constant__ CUtensorMap map_dy,
+                  const __grid_constant__ CUtensorMap map_x3,
+                  const __grid_constant__ CUtensorMap map_dy3,
+                  const __grid_constant__ CUtensorMap map_dy3h, int grouped,
+                  float *__restrict__ m_out,
                   float *__restrict__ v_out, long long ldmv, int tokens, int d_in, int d_out,
                   int split_from, int num_items, float a, float b, unsigned *status) {
     using G = Geo<CTAS>;
@@ -422,12 +445,20 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     const uint32_t sb = sa + G::A_STAGE_BYTES;
                     // out-of-range parts of a box are zero-filled and still counted
                     if (rank == 0) mbar_arrive_expect_tx(full0 + (uint32_t)stage * 8u, stage_tx);
+                    if (grouped) {
+                        // d_in, d_out multiples of 64: one operation per operand
+                        tma_load_3d<CTAS>(sa, &map_x3, kb * BK, m0 / GROUP, bar);
+                        tma_load_3d<CTAS>(sb, b_boxes == G::B_BOXES ? &map_dy3 : &map_dy3h, kb * BK,
+                                          n0 / GROUP, bar);
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < G::A_BOXES; ++j)
-                        tma_load_2d<CTAS>(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK, bar);
-                    for (int j = 0; j < b_boxes; ++j)
-                        tma_load_2d<CTAS>(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK,
-                                          bar);
+                        for (int j = 0; j < G::A_BOXES; ++j)
+                            tma_load_2d<CTAS>(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK,
+                                              bar);
+                        for (int j = 0; j < b_boxes; ++j)
+                            tma_load_2d<CTAS>(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK,
+                                              bar);
+                    }
                     armed |= 1u << stage;
                     last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == STAGES) {
@@ -648,6 +679,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 EncodeTiledFn g_encode = nullptr;
 bool g_attr_set = false;
 int g_variant = 0;  // 0 = not chosen yet, 1 = one-CTA tiles, 2 = CTA pairs
+bool g_no_grouped = false;
 
 // 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
 bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void *ptr,
@@ -659,6 +691,22 @@ bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// 3-D view of a row-major [tokens, d] bf16 matrix with d a multiple of 64:
+// {64 features (contiguous), tokens (pitch ld), d/64 groups (128 bytes apart)}; a box takes
+// 64 features x box_tokens x box_groups and lands group after group, 8192 bytes each.
+bool encode_grouped(CUtensorMap *map, const void *ptr, uint64_t d, uint64_t tokens, uint64_t ld,
+                    uint32_t box_tokens, uint32_t box_groups) {
+    cuuint64_t dims[3] = {GROUP, tokens, d / GROUP};
+    cuuint64_t strides[2] = {ld * 2, GROUP * 2};
+    cuuint32_t box[3] = {GROUP, box_tokens, box_groups};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims,
+                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -685,6 +733,8 @@ cudaError_t wgrad_fold_setup(const char **msg) {
         // ADAMA_WGRAD_CTAS=1 selects the one-CTA tiling (for comparisons); default: pairs
         const char *env = getenv("ADAMA_WGRAD_CTAS");
         g_variant = (env && env[0] == '1') ? 1 : 2;
+        const char *ng = getenv("ADAMA_WGRAD_NO_GROUPED");
+        g_no_grouped = ng && ng[0] == '1';
     }
     return cudaSuccess;
 }
@@ -711,6 +761,16 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
               encode_2d(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.dY, (uint64_t)p.d_out,
                         (uint64_t)p.tokens, (uint64_t)p.ldy, GROUP, BK,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    // grouped loads need whole 64-feature groups in both operands (CTA-pair kernel only)
+    CUtensorMap map_x3 = map_x, map_dy3 = map_dy, map_dy3h = map_dy;
+    int grouped = (g_variant == 2 && p.d_in % GROUP == 0 && p.d_out % GROUP == 0 && !g_no_grouped) ? 1 : 0;
+    if (ok && grouped)
+        ok = encode_grouped(&map_x3, p.X, (uint64_t)p.d_in, (uint64_t)p.tokens, (uint64_t)p.ldx, BK,
+                            Geo<2>::A_BOXES) &&
+             encode_grouped(&map_dy3, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens, (uint64_t)p.ldy,
+                            BK, Geo<2>::B_BOXES) &&
+             encode_grouped(&map_dy3h, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens,
+                            (uint64_t)p.ldy, BK, Geo<2>::B_BOXES / 2);
     if (!ok) {
         *msg = "cuTensorMapEncodeTiled rejected a tensor";
         return cudaErrorInvalidValue;
@@ -731,8 +791,8 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     const int groups = items < max_groups ? items : max_groups;
     if (g_variant == 1) {
         wgrad_fold_kernel<1><<<groups, NUM_THREADS, Geo<1>::SMEM_BYTES, p.stream>>>(
-            map_x, map_dy, p.m, p.v, (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from,
-            items, p.c.a, p.c.b, p.status);
+            map_x, map_dy, map_x3, map_dy3, map_dy3h, 0, p.m, p.v, (long long)p.ldmv, p.tokens,
+            p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status);
         return cudaGetLastError();
     }
     cudaLaunchConfig_t cfg = {};
@@ -747,7 +807,8 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, p.m, p.v,
+    return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_x3, map_dy3, map_dy3h,
+                              grouped, p.m, p.v,
                               (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
                               p.c.a, p.c.b, p.status);
 }
