@@ -54,7 +54,10 @@ namespace {
 #define ADAMA_WGRAD_STAGES 6  // shared-memory ring depth of the CTA-pair kernel (build-time tunable)
 #endif
 constexpr int BN = 256;     // tile columns (d_out direction) = UMMA N
-constexpr int BK = 64;      // tokens per pipeline stage
+#ifndef ADAMA_WGRAD_BK
+#define ADAMA_WGRAD_BK 64
+#endif
+constexpr int BK = ADAMA_WGRAD_BK;  // tokens per pipeline stage
 constexpr int UMMA_K = 16;  // tokens per tcgen05.mma (bf16)
 constexpr int GROUP = 64;   // features per 128-byte swizzled row
 constexpr int BOX_BYTES = GROUP * BK * 2;               // 8192
@@ -67,7 +70,7 @@ constexpr int EPI_BYTES = EPI_WARPS * EPI_BUF_BYTES;
 constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
-constexpr int MAX_STAGES = 6;
+constexpr int MAX_STAGES = 12;
 constexpr int SMEM_BAR_BYTES = 256;
 
 // Per-variant geometry: CTAS = CTAs cooperating on one tile (1 or 2).
@@ -81,7 +84,7 @@ struct Geo {
     static constexpr int A_STAGE_BYTES = A_BOXES * BOX_BYTES;
     static constexpr int B_STAGE_BYTES = B_BOXES * BOX_BYTES;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KB or 32 KB
-    static constexpr int STAGES = CTAS == 1 ? 4 : ADAMA_WGRAD_STAGES;
+    static constexpr int STAGES = CTAS == 1 ? 4 * 64 / BK : ADAMA_WGRAD_STAGES;
     static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
     static constexpr int SMEM_BYTES = SMEM_BAR_OFF + SMEM_BAR_BYTES + 1024;  // + alignment slack
