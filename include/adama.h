@@ -212,6 +212,24 @@ ADAMA_API adama_status adama_apply_allreduced(adama_ctx *ctx, float *w, float *m
 ADAMA_API adama_status adama_apply_sharded(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                            double lr, int world_size, void *cuda_stream);
 
+/* adama_apply_sharded with the exchange fused into the kernel: no separate reduce-scatter or
+ * all-gather.  w_peers, m_peers, v_peers are HOST arrays of world_size device pointers: entry
+ * q is rank q's full-size buffer (n fp32 elements), mapped into this process's address space
+ * (peer access over NVLink: IPC handles or symmetric memory; entry `rank` is the local one).
+ * This rank's launch reads shard `rank` (elements [rank*n/R, (rank+1)*n/R)) of every rank's m
+ * and v with plain loads, sums them in rank order, updates its shard of w as
+ * adama_apply_sharded does, and writes: the un-normalised sums into its own m, v shard, zeros
+ * into that shard of every other rank's m, v, and the new weights into that shard of every
+ * rank's w.  Shard r of all buffers is touched by rank r's launch only, and the kernel never
+ * waits for a peer.  The CALLER orders it against the folds: every rank has finished folding
+ * before the first of these launches starts, and none folds (or reads w) again before all of
+ * them have finished.  n must be a multiple of 4*world_size, all buffers 16-byte aligned,
+ * world_size <= 16.  Errors: INVALID_ARG, BAD_STATE, MISALIGNED, UNSUPPORTED, CUDA. */
+ADAMA_API adama_status adama_apply_sharded_peers(adama_ctx *ctx, float *const *w_peers,
+                                                 float *const *m_peers, float *const *v_peers,
+                                                 int world_size, int rank, size_t n, double lr,
+                                                 void *cuda_stream);
+
 /* ---- host-buffer variants (same arithmetic, copies included) --------------------------- */
 
 /* adama_fold with the gradient in HOST memory (pinned memory for full copy

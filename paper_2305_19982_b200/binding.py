@@ -17,7 +17,7 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
     "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
@@ -84,6 +84,8 @@ def load_library() -> ctypes.CDLL:
                                    ctypes.POINTER(vp), ctypes.POINTER(sz), ci, vp]
     L.adama_apply_multi.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
                                     ctypes.POINTER(sz), ci, dbl, vp]
+    L.adama_apply_sharded_peers.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                            ctypes.POINTER(vp), ci, ci, sz, dbl, vp]
     L.adama_bias_grad_fold.argtypes = [vp, vp, ci, ci, i64, vp, vp, vp]
     L.adama_fold_host.argtypes = [vp, vp, ci, vp, vp, sz, vp, sz, vp]
     L.adama_linear_wgrad_fold_host.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, i64, vp, sz, vp]
@@ -241,6 +243,17 @@ class AdamA:
                                         _dev_ptr(m, torch.float32, "m"),
                                         _dev_ptr(v, torch.float32, "v"), n, float(lr),
                                         _stream_ptr(self.device)))
+
+    def apply_sharded_peers(self, w_ptrs, m_ptrs, v_ptrs, rank: int, n: int, lr: float) -> None:
+        """adama_apply_sharded_peers: lists of raw device pointers (ints), one per rank, to the
+        peer-mapped full-size w, m, v buffers; `rank` is this process's index."""
+        world = len(w_ptrs)
+        if len(m_ptrs) != world or len(v_ptrs) != world:
+            raise ValueError("pointer lists must have equal length")
+        arr = lambda ps: (ctypes.c_void_p * world)(*[int(p) for p in ps])
+        self._check(self._L.adama_apply_sharded_peers(
+            self._h, arr(w_ptrs), arr(m_ptrs), arr(v_ptrs), world, int(rank), int(n), float(lr),
+            _stream_ptr(self.device)))
 
     def bias_grad_fold(self, dY: torch.Tensor, m: torch.Tensor, v: torch.Tensor) -> None:
         """adama_bias_grad_fold: dY [tokens, d_out] bf16 (unit stride in the last dim), m, v [d_out]."""

@@ -279,6 +279,39 @@ adama_status adama_apply_sharded(adama_ctx *ctx, float *w, float *m, float *v, s
     return apply_impl(ctx, w, m, v, n, lr, world_size, true, cuda_stream);
 }
 
+adama_status adama_apply_sharded_peers(adama_ctx *ctx, float *const *w_peers, float *const *m_peers,
+                                       float *const *v_peers, int world_size, int rank, size_t n,
+                                       double lr, void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (world_size < 1 || rank < 0 || rank >= world_size || !w_peers || !m_peers || !v_peers)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply_sharded_peers: bad world size, rank or list");
+    if (world_size > adama::kMaxPeers)
+        return fail(ctx, ADAMA_ERR_UNSUPPORTED, "apply_sharded_peers: more than 16 peers");
+    if (!isfinite(lr)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply_sharded_peers: lr is not finite");
+    if (ctx->t < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "apply_sharded_peers: no mini-batch has been started");
+    if (n % (4 * (size_t)world_size))
+        return fail(ctx, ADAMA_ERR_UNSUPPORTED,
+                    "apply_sharded_peers: n must be a multiple of 4*world_size (pad the buffers)");
+    for (int q = 0; q < world_size; ++q) {
+        if (n > 0 && (!w_peers[q] || !m_peers[q] || !v_peers[q]))
+            return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply_sharded_peers: null peer pointer");
+        if (!aligned_to(w_peers[q], 16) || !aligned_to(m_peers[q], 16) || !aligned_to(v_peers[q], 16))
+            return fail(ctx, ADAMA_ERR_MISALIGNED, "apply_sharded_peers: buffers must be 16-byte aligned");
+    }
+    if (n == 0) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    const adama::ApplyConstants c =
+        adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr,
+                                    world_size, true, ctx->weight_decay);
+    cudaError_t e = adama::launch_apply_sharded_peers(w_peers, m_peers, v_peers, world_size, rank, n,
+                                                      c, ctx->sm_count,
+                                                      static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "apply_sharded_peers launch", e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
 adama_status adama_bias_grad_fold(adama_ctx *ctx, const void *dY, int tokens, int d_out,
                                   int64_t ldy, float *m, float *v, void *cuda_stream) {
     if (!ctx) return ADAMA_ERR_INVALID_ARG;

@@ -57,6 +57,12 @@ cudaError_t launch_fold_multi(const void *const *g, adama_dtype gdt, float *cons
 cudaError_t launch_apply_multi(float *const *w, float *const *m, float *const *v, const size_t *n,
                                int count, ApplyConstants c, int sm_count, cudaStream_t stream);
 
+// fused reduce-scatter + sharded apply + all-gather over peer-mapped buffers (peer_apply.cu)
+constexpr int kMaxPeers = 16;
+cudaError_t launch_apply_sharded_peers(float *const *w, float *const *m, float *const *v, int world,
+                                       int rank, size_t n, ApplyConstants c, int sm_count,
+                                       cudaStream_t stream);
+
 // bias gradient (column sums of dY) + fold (bias_grad.cu)
 cudaError_t launch_bias_grad_fold(const void *dY, int tokens, int d_out, int64_t ldy, float *m,
                                   float *v, FoldConstants c, cudaStream_t stream);

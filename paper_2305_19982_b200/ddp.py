@@ -66,3 +66,42 @@ def reduce_scatter_apply_allgather(opt, w: torch.Tensor, m: torch.Tensor, v: tor
         parts = [torch.empty_like(wf[lo:hi]) for _ in range(world)]
         dist.all_gather(parts, wf[lo:hi].clone(), group=group)
         wf.copy_(torch.cat(parts))
+
+
+class PeerMappedStates:
+    """w, m, v of one replica allocated in torch symmetric memory, so that every rank can
+    address every other rank's buffers (NVLink peer access) and the whole end-of-mini-batch
+    exchange is ONE kernel per rank (`AdamA.apply_sharded_peers`): no reduce-scatter, no
+    all-gather.  The two barriers around it are the ordering the kernel asks of its caller.
+
+    Written against torch.distributed._symmetric_memory; this repository's tests exercise the
+    kernel with all ranks' buffers on one GPU (tests/test_gpu_ddp.py), not this allocation
+    path on several GPUs.
+    """
+
+    def __init__(self, n: int, device, group=None):
+        import torch.distributed._symmetric_memory as symm_mem
+        self.group = group if group is not None else dist.group.WORLD
+        self.world = dist.get_world_size(self.group)
+        self.rank = dist.get_rank(self.group)
+        if n % (4 * self.world):
+            raise ValueError("n must be a multiple of 4 * world size (pad the flat buffer)")
+        self.n = n
+        self._bufs, self._handles = {}, {}
+        for name in ("w", "m", "v"):
+            t = symm_mem.empty(n, dtype=torch.float32, device=device)
+            self._handles[name] = symm_mem.rendezvous(t, self.group)
+            self._bufs[name] = t
+        self.m.zero_()
+        self.v.zero_()
+
+    w = property(lambda self: self._bufs["w"])
+    m = property(lambda self: self._bufs["m"])
+    v = property(lambda self: self._bufs["v"])
+
+    def exchange_and_apply(self, opt, lr: float) -> None:
+        h = self._handles
+        h["m"].barrier()          # every rank has finished folding into its m, v
+        opt.apply_sharded_peers(list(h["w"].buffer_ptrs), list(h["m"].buffer_ptrs),
+                                list(h["v"].buffer_ptrs), self.rank, self.n, lr)
+        h["m"].barrier()          # every shard has been written everywhere

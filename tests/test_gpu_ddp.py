@@ -119,3 +119,48 @@ def test_sharded_apply_equals_single_device(R, N):
             assert rel_l2(f64(v[r][lo:hi]), R * R * wl.BETA2 * single.v[lo:hi]) <= TOL
     for o in opts:
         o.close()
+
+
+@pytest.mark.parametrize("R,N", [(2, 2), (4, 1), (8, 1)])
+def test_fused_peer_exchange_apply_equals_single_device(R, N):
+    """adama_apply_sharded_peers: reduce-scatter + update + all-gather in one kernel over
+    peer-mapped buffers.  The R ranks' buffers all live on this one GPU and the R launches run
+    one after the other (the kernel never waits for a peer, so this is a faithful emulation):
+    every rank must end with the single-device weights for N*R micro-batches, keep the
+    un-normalised sums for its own shard only, and hold zeros elsewhere."""
+    n, steps = 4 * R * 1031, 3
+    k = n // R
+    w0 = wl.normal((n,), 0.02, torch.float32, 21)
+    single = AdamAOracle(f64(w0))
+    opts = [adama.AdamA() for _ in range(R)]
+    w = [w0.cuda() for _ in range(R)]
+    m = [torch.zeros(n, device="cuda") for _ in range(R)]
+    v = [torch.zeros(n, device="cuda") for _ in range(R)]
+    ptrs = lambda ts: [t.data_ptr() for t in ts]
+    for step in range(steps):
+        single.begin_minibatch(N * R)
+        for r in range(R):
+            opts[r].begin_minibatch(N)
+            for i in range(N):
+                g = wl.normal((n,), 1e-2, torch.float32, 3000 * step + 10 * r + i + 5)
+                opts[r].fold(g.cuda(), m[r], v[r])
+                single.fold(f64(g))
+        torch.cuda.synchronize()                       # "all ranks have finished folding"
+        for r in range(R):
+            opts[r].apply_sharded_peers(ptrs(w), ptrs(m), ptrs(v), r, n, wl.LR)
+        torch.cuda.synchronize()                       # "all exchanges have finished"
+        single.update(wl.LR)
+        for r in range(R):
+            lo, hi = r * k, (r + 1) * k
+            assert rel_l2(f64(w[r]), single.theta) <= TOL
+            assert torch.equal(w[r], w[0])
+            assert rel_l2(f64(m[r][lo:hi]), R * wl.BETA1 * single.m[lo:hi]) <= TOL
+            assert rel_l2(f64(v[r][lo:hi]), R * R * wl.BETA2 * single.v[lo:hi]) <= TOL
+            mask = torch.ones(n, dtype=torch.bool, device="cuda")
+            mask[lo:hi] = False
+            assert not bool(m[r][mask].any()) and not bool(v[r][mask].any())
+    with pytest.raises(adama.AdamAError) as e:
+        opts[0].apply_sharded_peers(ptrs(w), ptrs(m), ptrs(v), 0, n - 4, wl.LR)
+    assert e.value.status == adama.Status.ERR_UNSUPPORTED
+    for o in opts:
+        o.close()
