@@ -317,6 +317,13 @@ ADAMA_API adama_status adama_set_weight_decay(adama_ctx *ctx, double weight_deca
  * expired; m and v of that call are incomplete) or ADAMA_ERR_CUDA. */
 ADAMA_API adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream);
 
+/* Test hook: writes {code, wait, tile} into the device status block exactly as a kernel whose
+ * bounded wait expired would, so that the host side of the time-out path (adama_sync_status:
+ * report, message, clearing, continued use of the context) can be exercised without making
+ * any kernel wait in vain.  Synchronises `cuda_stream`. */
+ADAMA_API adama_status adama_debug_set_status(adama_ctx *ctx, unsigned code, unsigned wait,
+                                              unsigned tile, void *cuda_stream);
+
 /* Message for the most recent non-OK status returned on this context ("" if
  * none).  The pointer stays valid until the next call on the context. */
 ADAMA_API const char *adama_last_error(const adama_ctx *ctx);

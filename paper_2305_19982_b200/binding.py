@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
-    "adama_sync_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
+    "adama_sync_status", "adama_debug_set_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
     "adama_host_constants_allreduced", "adama_host_constants_sharded",
     "adama_version",
 ]
@@ -98,6 +98,7 @@ def load_library() -> ctypes.CDLL:
     L.adama_get_n_micro.argtypes = [vp]
     L.adama_set_weight_decay.argtypes = [vp, dbl]
     L.adama_sync_status.argtypes = [vp, vp]
+    L.adama_debug_set_status.argtypes = [vp, ctypes.c_uint, ctypes.c_uint, ctypes.c_uint, vp]
     L.adama_last_error.argtypes = [vp]
     L.adama_last_error.restype = ctypes.c_char_p
     L.adama_launch_count.argtypes = [vp]
@@ -387,6 +388,11 @@ class AdamA:
         """Waits for the current stream and raises AdamAError(ERR_TIMEOUT) if a bounded
         device-side wait expired."""
         self._check(self._L.adama_sync_status(self._h, _stream_ptr(self.device)))
+
+    def debug_set_status(self, code: int, wait: int = 0, tile: int = 0) -> None:
+        """adama_debug_set_status (test hook for the time-out reporting path)."""
+        self._check(self._L.adama_debug_set_status(self._h, code, wait, tile,
+                                                   _stream_ptr(self.device)))
 
     @property
     def launch_count(self) -> int:

@@ -549,6 +549,18 @@ adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream) {
     return ADAMA_OK;
 }
 
+adama_status adama_debug_set_status(adama_ctx *ctx, unsigned code, unsigned wait, unsigned tile,
+                                    void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const unsigned words[4] = {code, wait, tile, 0};
+    cudaError_t e = cudaMemcpyAsync(ctx->status_dev, words, sizeof(words), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);  // `words` lives on this stack frame
+    if (e != cudaSuccess) return cuda_fail(ctx, "debug_set_status", e);
+    return ADAMA_OK;
+}
+
 const char *adama_last_error(const adama_ctx *ctx) { return ctx ? ctx->err : ""; }
 
 int64_t adama_launch_count(const adama_ctx *ctx) { return ctx ? ctx->launches : -1; }

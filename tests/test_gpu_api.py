@@ -76,3 +76,55 @@ def test_host_staging_checks():
     small = torch.empty(1024, dtype=torch.uint8, device="cuda")
     assert _err(opt.fold_host, g, m, m.clone(), small) == Status.ERR_INVALID_ARG
     opt.close()
+
+
+def test_timeout_report_path_without_a_waiting_kernel():
+    """The host side of the bounded-wait design: a status block that says "a wait expired" is
+    reported once as ERR_TIMEOUT with the wait and tile in the message, cleared, and the
+    context keeps working.  The record is planted by the test hook; no kernel is made to wait."""
+    import adama_workloads as wl
+    opt = adama.AdamA()
+    opt.sync_status()                                   # clean
+    opt.debug_set_status(1, wait=3, tile=17)
+    with pytest.raises(adama.AdamAError) as e:
+        opt.sync_status()
+    assert e.value.status == Status.ERR_TIMEOUT and "wait 3" in str(e.value) and "tile 17" in str(e.value)
+    opt.sync_status()                                   # cleared by the report
+    opt.begin_minibatch(1)
+    X = wl.small_integers((64, 128), 2, torch.bfloat16, 1).cuda()
+    dY = wl.small_integers((64, 256), 2, torch.bfloat16, 2).cuda()
+    m = torch.zeros(128, 256, device="cuda")
+    v = torch.zeros(128, 256, device="cuda")
+    opt.linear_wgrad_fold(X, dY, m, v)                  # the context is still usable
+    opt.sync_status()
+    assert torch.allclose(m, (1 - 0.9) * (X.float().t() @ dY.float()), rtol=1e-6)
+    opt.close()
+
+
+def test_checkpoint_resume_is_bit_identical():
+    """State = w, m, v (stored decayed after apply) + the step counter: a new context restored
+    with set_step continues exactly as the uninterrupted run."""
+    import adama_workloads as wl
+    n, N = 50_000, 2
+
+    def run(total_steps, resume_after=None):
+        opt = adama.AdamA()
+        w = wl.normal((n,), 0.02, torch.float32, 5).cuda()
+        m, v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+        for step in range(total_steps):
+            if resume_after is not None and step == resume_after:
+                saved = (w.clone(), m.clone(), v.clone(), opt.step)
+                opt.close()
+                opt = adama.AdamA()                     # "new process": fresh context
+                w, m, v = saved[0], saved[1], saved[2]
+                opt.set_step(saved[3])
+            opt.begin_minibatch(N)
+            for i in range(N):
+                opt.fold(wl.normal((n,), 1e-2, torch.bfloat16, 100 * step + i).cuda(), m, v)
+            opt.apply(w, m, v, 1e-3)
+        opt.close()
+        return w, m, v
+
+    a = run(4)
+    b = run(4, resume_after=2)
+    assert all(torch.equal(x, y) for x, y in zip(a, b))

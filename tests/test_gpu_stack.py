@@ -97,3 +97,17 @@ def test_gpt2xl_full_stack_sampled():
 def test_llama7b_two_blocks_sampled():
     stack = llama7b_stack(2)
     _sampled_stack(stack, wl.CONFIG5_TOKENS, 1, 5, 40)
+
+
+def test_llama7b_full_stack_sampled():
+    """All 32 blocks x 7 linears (6.476 B parameters, 77.7 GB of fp32 state), 4096 tokens, one
+    micro-batch, 10 sampled entries per layer, in the launch configuration the bench times."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100 * (1 << 30):
+        pytest.skip("needs ~90 GB of free device memory")
+    torch.cuda.empty_cache()
+    stack = llama7b_stack(wl.CONFIG5_BLOCKS)
+    assert stack.n_params == 32 * (4 * 4096 * 4096 + 3 * 4096 * 11008)
+    _sampled_stack(stack, wl.CONFIG5_TOKENS, 1, 5, 10)
+    del stack
+    torch.cuda.empty_cache()
