@@ -365,6 +365,7 @@ def run_ours(args):
     optA.close()
     optB.close()
     if dist is not None:
+        dist.barrier()  # rank 0 may still be printing; leave the group together
         dist.destroy_process_group()
 
 
