@@ -153,6 +153,15 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
 ADAMA_API adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                    double lr, void *cuda_stream);
 
+/* adama_apply that also writes the updated weights rounded to bf16 (round to nearest even)
+ * into w_bf16_out (n bf16 elements, device): the copy a mixed-precision forward pass reads,
+ * produced in the same pass (26 B/param) instead of by a separate cast (24 + 6).  The fp32
+ * w stays the master copy; w, m, v results are bit-identical to adama_apply.
+ * Errors: as adama_apply, plus INVALID_ARG (null output), MISALIGNED. */
+ADAMA_API adama_status adama_apply_bf16_copy(adama_ctx *ctx, float *w, float *m, float *v,
+                                             void *w_bf16_out, size_t n, double lr,
+                                             void *cuda_stream);
+
 /* The bias of the same linear layer: its raw micro-batch gradient is the column sum of dY,
  *     g[q] = sum_{tau < tokens} dY[tau,q],   m[q] += a*g[q],   v[q] += b*g[q]^2
  * (Algorithm 2, inner loop body; the sum over tokens is completed on-chip, by a cluster of

@@ -17,7 +17,7 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
+    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_bf16_copy", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
     "adama_sync_status", "adama_debug_set_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
@@ -75,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     L.adama_fold.argtypes = [vp, vp, ci, vp, vp, sz, vp]
     L.adama_linear_wgrad_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp]
     L.adama_apply.argtypes = [vp, vp, vp, vp, sz, dbl, vp]
+    L.adama_apply_bf16_copy.argtypes = [vp, vp, vp, vp, vp, sz, dbl, vp]
     L.adama_apply_allreduced.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
     L.adama_host_constants_allreduced.argtypes = [ctypes.POINTER(_Config), ci, i64, dbl, ci,
                                                   ctypes.POINTER(ctypes.c_float)]
@@ -298,6 +299,19 @@ class AdamA:
             raise ValueError("w, m, v must have the same number of elements")
         self._check(self._L.adama_apply_multi(self._h, ws.ptrs, ms.ptrs, vs.ptrs, ws.ns, len(ws),
                                               float(lr), _stream_ptr(self.device)))
+
+    def apply_bf16_copy(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
+                        w_bf16: torch.Tensor, lr: float) -> None:
+        """adama_apply_bf16_copy: apply, and write the updated weights to `w_bf16` as bf16."""
+        if not (w.is_contiguous() and m.is_contiguous() and v.is_contiguous() and w_bf16.is_contiguous()):
+            raise ValueError("apply needs contiguous tensors")
+        n = w.numel()
+        if m.numel() != n or v.numel() != n or w_bf16.numel() != n:
+            raise ValueError("w, m, v, w_bf16 must have the same number of elements")
+        self._check(self._L.adama_apply_bf16_copy(
+            self._h, _dev_ptr(w, torch.float32, "w"), _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), _dev_ptr(w_bf16, torch.bfloat16, "w_bf16"), n,
+            float(lr), _stream_ptr(self.device)))
 
     def apply_allreduced(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float,
                          world_size: int) -> None:

@@ -248,7 +248,8 @@ adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *
 }
 
 static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
-                               int world, bool sharded, void *cuda_stream) {
+                               int world, bool sharded, void *cuda_stream,
+                               void *w_bf16_out = nullptr) {
     adama_status st = check_apply_args(ctx, w, m, v, n, lr);
     if (st != ADAMA_OK) return st;
     if (world < 1) return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply: world_size must be >= 1");
@@ -258,10 +259,19 @@ static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, siz
                                                           ctx->cfg.eps, ctx->t, lr, world, sharded,
                                                           ctx->weight_decay);
     cudaError_t e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
-                                        static_cast<cudaStream_t>(cuda_stream));
+                                        static_cast<cudaStream_t>(cuda_stream), w_bf16_out);
     if (e != cudaSuccess) return cuda_fail(ctx, "apply launch", e);
     ctx->launches += 1;
     return ADAMA_OK;
+}
+
+adama_status adama_apply_bf16_copy(adama_ctx *ctx, float *w, float *m, float *v, void *w_bf16_out,
+                                   size_t n, double lr, void *cuda_stream) {
+    if (ctx && n > 0 && !w_bf16_out)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "apply_bf16_copy: null bf16 output");
+    if (ctx && !aligned_to(w_bf16_out, 2))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "apply_bf16_copy: bf16 output not 2-byte aligned");
+    return apply_impl(ctx, w, m, v, n, lr, 1, false, cuda_stream, w_bf16_out);
 }
 
 adama_status adama_apply(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,

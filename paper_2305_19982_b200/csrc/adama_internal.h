@@ -45,8 +45,9 @@ enum DeviceErr : unsigned { kDevOk = 0, kDevTimeout = 1 };
 // streaming kernels (fold_apply.cu)
 cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, size_t n,
                         FoldConstants c, int sm_count, cudaStream_t stream);
+// w_bf16_out (may be null): n bf16 elements that receive the updated weights, rounded to nearest
 cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants c, int sm_count,
-                         cudaStream_t stream);
+                         cudaStream_t stream, void *w_bf16_out = nullptr);
 
 // multi-tensor forms (multi_tensor.cu): up to kMultiMax tensors per launch, each shorter than
 // 2^32 * 4096 elements in total blocks

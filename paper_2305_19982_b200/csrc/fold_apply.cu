@@ -158,10 +158,18 @@ __device__ __forceinline__ void apply1(float &w, float &m, float &v, const Apply
     v = fmaf(v, c.beta2_hi, v * c.beta2_lo);
 }
 
-template <int UNROLL>
+// two fp32 -> packed bf16x2, round to nearest even
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const unsigned *>(&p);
+}
+
+// COPY: also write the updated weights rounded to bf16 (the copy a mixed-precision forward
+// pass reads), 2 B/param on top of the 24, instead of a separate cast pass of 6 B/param.
+template <int UNROLL, bool COPY>
 __global__ void __launch_bounds__(kThreads, kApplyCtasPerSm)
-apply_vec_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict__ v, size_t n4,
-                 size_t n, ApplyConstants c) {
+apply_vec_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict__ v,
+                 __nv_bfloat16 *__restrict__ w_bf16, size_t n4, size_t n, ApplyConstants c) {
     float4 *w4 = reinterpret_cast<float4 *>(w);
     float4 *m4 = reinterpret_cast<float4 *>(m);
     float4 *v4 = reinterpret_cast<float4 *>(v);
@@ -188,6 +196,9 @@ apply_vec_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict
                 st_stream(w4 + i, ww[u]);
                 st_stream(m4 + i, mm[u]);
                 st_stream(v4 + i, vv[u]);
+                if (COPY)
+                    reinterpret_cast<uint2 *>(w_bf16)[i] =
+                        make_uint2(pack_bf16x2(ww[u].x, ww[u].y), pack_bf16x2(ww[u].z, ww[u].w));
             }
         }
     }
@@ -198,12 +209,13 @@ apply_vec_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict
         w[i] = wi;
         m[i] = mi;
         v[i] = vi;
+        if (COPY) w_bf16[i] = __float2bfloat16_rn(wi);
     }
 }
 
 __global__ void __launch_bounds__(kThreads)
-apply_scalar_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict__ v, size_t n,
-                    ApplyConstants c) {
+apply_scalar_kernel(float *__restrict__ w, float *__restrict__ m, float *__restrict__ v,
+                    __nv_bfloat16 *__restrict__ w_bf16, size_t n, ApplyConstants c) {
     for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n;
          i += (size_t)gridDim.x * kThreads) {
         float wi = w[i], mi = m[i], vi = v[i];
@@ -211,6 +223,7 @@ apply_scalar_kernel(float *__restrict__ w, float *__restrict__ m, float *__restr
         w[i] = wi;
         m[i] = mi;
         v[i] = vi;
+        if (w_bf16) w_bf16[i] = __float2bfloat16_rn(wi);
     }
 }
 
@@ -257,16 +270,20 @@ cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, s
 }
 
 cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants c, int sm_count,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, void *w_bf16_out) {
+    __nv_bfloat16 *wb = static_cast<__nv_bfloat16 *>(w_bf16_out);
     if (n == 0) return cudaSuccess;
     constexpr int U = ADAMA_APPLY_UNROLL;
     const size_t n4 = n / 4;
-    if (aligned(w, 16) && aligned(m, 16) && aligned(v, 16)) {
+    if (aligned(w, 16) && aligned(m, 16) && aligned(v, 16) && (!wb || aligned(wb, 8))) {
         unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count, kApplyCtasPerSm);
-        apply_vec_kernel<U><<<grid, kThreads, 0, stream>>>(w, m, v, n4, n, c);
+        if (wb)
+            apply_vec_kernel<U, true><<<grid, kThreads, 0, stream>>>(w, m, v, wb, n4, n, c);
+        else
+            apply_vec_kernel<U, false><<<grid, kThreads, 0, stream>>>(w, m, v, nullptr, n4, n, c);
     } else {
         unsigned grid = grid_for(n, kThreads, sm_count);
-        apply_scalar_kernel<<<grid, kThreads, 0, stream>>>(w, m, v, n, c);
+        apply_scalar_kernel<<<grid, kThreads, 0, stream>>>(w, m, v, wb, n, c);
     }
     return cudaGetLastError();
 }

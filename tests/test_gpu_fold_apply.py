@@ -204,3 +204,28 @@ def test_decoupled_weight_decay_extension():
         opt.set_weight_decay(-1.0)
     for o in (opt, plain, zero):
         o.close()
+
+
+@pytest.mark.parametrize("n,offset", [(1_000_003, 0), (4099, 0), (10_007, 1), (5, 0)])
+def test_apply_with_bf16_copy(n, offset):
+    """The bf16 copy is the round-to-nearest-even of the fp32 result, and w, m, v are the same
+    bits as plain apply gives (vector and scalar paths)."""
+    g = wl.normal((n,), 1e-2, torch.float32, 77).cuda()
+    res = []
+    for copy in (False, True):
+        opt = adama.AdamA()
+        opt.begin_minibatch(1)
+        w = Guarded(n, offset=offset).fill(wl.normal((n,), 0.02, torch.float32, 78).cuda())
+        m, v = Guarded(n, offset=offset).zero(), Guarded(n, offset=offset).zero()
+        wb = Guarded(n, dtype=torch.bfloat16, offset=offset)
+        opt.fold(g, m.view, v.view)
+        if copy:
+            opt.apply_bf16_copy(w.view, m.view, v.view, wb.view, wl.LR)
+            assert torch.equal(wb.view, w.view.to(torch.bfloat16))
+        else:
+            opt.apply(w.view, m.view, v.view, wl.LR)
+        for b in (w, m, v, wb):
+            b.check()
+        res.append((w.view.clone(), m.view.clone(), v.view.clone()))
+        opt.close()
+    assert all(torch.equal(a, b) for a, b in zip(*res))
