@@ -5,7 +5,7 @@
 // per thread, grid sized as a multiple of the SM count with a grid-stride loop.
 #include <cuda_bf16.h>
 
-#include "adama_internal.h"
+#include "adama_device.cuh"
 
 namespace adama {
 namespace {
@@ -84,12 +84,6 @@ __device__ __forceinline__ Grad4 load_grad4(const __nv_bfloat16 *g, size_t i4) {
 __device__ __forceinline__ float widen(float g) { return g; }
 __device__ __forceinline__ float widen(__nv_bfloat16 g) { return __bfloat162float(g); }
 
-// m += a*g ; v += b*g^2      (Algorithm 2: m += (1-beta1) g/N, v += (1-beta2) (g/N)^2)
-__device__ __forceinline__ void fold1(float g, float &m, float &v, float a, float b) {
-    m = fmaf(a, g, m);
-    v = fmaf(b * g, g, v);
-}
-
 template <typename G, int UNROLL>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 fold_vec_kernel(const G *__restrict__ grad, float *__restrict__ m, float *__restrict__ v,
@@ -145,17 +139,6 @@ fold_scalar_kernel(const G *__restrict__ grad, float *__restrict__ m, float *__r
         m[i] = mi;
         v[i] = vi;
     }
-}
-
-// w -= step * m / (sqrt(v*inv_bc2) + eps);  m *= beta1;  v *= beta2
-__device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
-    float denom = sqrtf(v * c.inv_bc2) + c.eps;  // IEEE sqrt
-    w = fmaf(-c.step, m / denom, w * c.w_keep);             // IEEE division
-    // beta = hi + lo: the small product is rounded first (its error is ~1e-15 relative to
-    // the result), then one fma rounds x*hi + x*lo once.  The other order would round
-    // x*hi first and lose the sub-ulp correction every time.
-    m = fmaf(m, c.beta1_hi, m * c.beta1_lo);
-    v = fmaf(v, c.beta2_hi, v * c.beta2_lo);
 }
 
 // two fp32 -> packed bf16x2, round to nearest even

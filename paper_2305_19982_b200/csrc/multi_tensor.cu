@@ -5,7 +5,7 @@
 // the kernel's parameter space, no device memory is allocated.
 #include <cuda_bf16.h>
 
-#include "adama_internal.h"
+#include "adama_device.cuh"
 
 namespace adama {
 namespace {
@@ -69,33 +69,22 @@ fold_multi_kernel(const __grid_constant__ MultiTable tab, float a, float b) {
                 float x[4];
                 load4(g + 4 * i, x);
                 float4 mm = reinterpret_cast<float4 *>(m)[i], vv = reinterpret_cast<float4 *>(v)[i];
-                mm.x = fmaf(a, x[0], mm.x); vv.x = fmaf(b * x[0], x[0], vv.x);
-                mm.y = fmaf(a, x[1], mm.y); vv.y = fmaf(b * x[1], x[1], vv.y);
-                mm.z = fmaf(a, x[2], mm.z); vv.z = fmaf(b * x[2], x[2], vv.z);
-                mm.w = fmaf(a, x[3], mm.w); vv.w = fmaf(b * x[3], x[3], vv.w);
+                fold1(x[0], mm.x, vv.x, a, b);
+                fold1(x[1], mm.y, vv.y, a, b);
+                fold1(x[2], mm.z, vv.z, a, b);
+                fold1(x[3], mm.w, vv.w, a, b);
                 reinterpret_cast<float4 *>(m)[i] = mm;
                 reinterpret_cast<float4 *>(v)[i] = vv;
             }
             for (size_t i = c4 * 4 + threadIdx.x; i < cnt; i += kThreads) {
-                const float x = widen(g[i]);
-                m[i] = fmaf(a, x, m[i]);
-                v[i] = fmaf(b * x, x, v[i]);
+                fold1(widen(g[i]), m[i], v[i], a, b);
             }
         } else {
             for (size_t i = threadIdx.x; i < cnt; i += kThreads) {
-                const float x = widen(g[i]);
-                m[i] = fmaf(a, x, m[i]);
-                v[i] = fmaf(b * x, x, v[i]);
+                fold1(widen(g[i]), m[i], v[i], a, b);
             }
         }
     }
-}
-
-__device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
-    const float denom = sqrtf(v * c.inv_bc2) + c.eps;
-    w = fmaf(-c.step, m / denom, w * c.w_keep);
-    m = fmaf(m, c.beta1_hi, m * c.beta1_lo);
-    v = fmaf(v, c.beta2_hi, v * c.beta2_lo);
 }
 
 __global__ void __launch_bounds__(kThreads)

@@ -10,7 +10,7 @@
 // The ranks must have finished folding before any of these launches starts and must not fold
 // again before all of them have finished; that ordering is the caller's (a barrier on the
 // host or between streams), so the kernel itself never waits for a peer.
-#include "adama_internal.h"
+#include "adama_device.cuh"
 
 namespace adama {
 namespace {
@@ -37,13 +37,6 @@ __device__ __forceinline__ void st4(float *p, float4 x) {
                  "f"(x.w)
                  : "memory");
 }
-__device__ __forceinline__ void apply1(float &w, float &m, float &v, const ApplyConstants &c) {
-    const float denom = sqrtf(v * c.inv_bc2) + c.eps;
-    w = fmaf(-c.step, m / denom, w * c.w_keep);
-    m = fmaf(m, c.beta1_hi, m * c.beta1_lo);
-    v = fmaf(v, c.beta2_hi, v * c.beta2_lo);
-}
-
 __global__ void __launch_bounds__(kThreads)
 apply_sharded_peers_kernel(const __grid_constant__ PeerTable tab, size_t lo4, size_t n4,
                            ApplyConstants c) {
