@@ -12,7 +12,7 @@
 // was measured first: the L2's reduction rate, about 2 TB/s of payload, stalled the
 // operand loads of the overlapped main loop; plain reads and writes do not.)
 //
-// Persistent kernel, 192 threads per CTA, CTAs working in pairs (a cluster of two on
+// Persistent kernel, 192 or 320 threads per CTA, CTAs working in pairs (a cluster of two on
 // the two SMs of a TPC, tcgen05 cta_group::2): a pair owns a 256x256 output tile,
 // each CTA its 128 rows.  Per 64-token stage a CTA loads its own 128 rows of X^T and
 // only HALF of the dY tile (128 of the 256 columns); the tensor cores of both SMs
@@ -20,8 +20,8 @@
 // instead of 96 for a lone 128x256 tile, and leaves room for a 6-stage ring.
 //   warp 0      TMA producer: operand tiles -> shared-memory ring (both CTAs)
 //   warp 1      MMA issuer (one thread of the pair's first CTA) + TMEM allocation
-//   warps 2..9  epilogue: two warps per TMEM lane quarter, one per half of the tile's
-//               columns (both CTAs)
+//   warps 2..   epilogue: one or two warps per TMEM lane quarter (4 or 8 warps, chosen per
+//               launch; with two, each takes half of the tile's columns), in both CTAs
 // The 512 TMEM columns hold two 128x256 fp32 accumulators per CTA, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  (A one-CTA variant, 128x256 tiles and a
 // 4-stage ring, is kept as a template instance for comparison.)
@@ -36,8 +36,7 @@
 // Synchronisation of a pair: the first CTA's "full" barrier of a stage counts the
 // bytes of both CTAs' loads; when the MMAs that read a stage retire, tcgen05.commit
 // arrives on the "empty" barrier of each CTA; the same for accumulator-full; the
-// sixteen epilogue warps of the pair arrive on the first CTA's accumulator-empty
-// barrier.  No load uses cluster multicast.
+// epilogue warps of both CTAs arrive on the first CTA's accumulator-empty barrier.  No load uses cluster multicast.
 //
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the kernel
 // records a code in the status block, all roles drain and leave, TMEM is freed.
@@ -64,10 +63,14 @@ constexpr int BOX_BYTES = GROUP * BK * 2;               // 8192
 constexpr int EPI_COLS = 32;                            // fp32 columns per epilogue chunk (128 B)
 constexpr int EPI_ROWS = 32;                            // one TMEM lane quarter
 constexpr int EPI_BUF_BYTES = EPI_ROWS * EPI_COLS * 4;  // 4096: one transposition buffer per warp
-constexpr int EPI_WARPS = 8;                            // 4 lane quarters x COL_SPLIT column parts
-constexpr int COL_SPLIT = EPI_WARPS / 4;
-constexpr int EPI_BYTES = EPI_WARPS * EPI_BUF_BYTES;
-constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
+// Epilogue warps: 4 (one per TMEM lane quarter) or 8 (two per quarter, each half of the tile's
+// columns), chosen per launch through the block size.  Measured: when tiles queue up behind
+// each other 4 warps disturb the overlapped main loop less (4096x11008: 274 vs 279 us); when
+// every CTA pair has a single tile its epilogue is fully exposed and 8 warps finish it sooner
+// (1600x1600: 41.8 vs 43.8 us).
+constexpr int MAX_EPI_WARPS = 8;
+constexpr int EPI_BYTES = MAX_EPI_WARPS * EPI_BUF_BYTES;
+constexpr int MAX_THREADS = 32 * (2 + MAX_EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
 constexpr int MAX_STAGES = 12;
@@ -371,7 +374,7 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
 }
 
 template <int CTAS>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(MAX_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   const __grid_constant__ CUtensorMap map_dy,
                   const __grid_constant__ CUtensorMap map_x3,
@@ -404,7 +407,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         }
         for (int s = 0; s < ACC_STAGES; ++s) {
             mbar_init(smem_u32(&bars->acc_full[s]), 1);
-            mbar_init(smem_u32(&bars->acc_empty[s]), EPI_WARPS * CTAS);
+            mbar_init(smem_u32(&bars->acc_empty[s]), (blockDim.x / 32 - 2) * CTAS);
         }
         mbar_init(smem_u32(&bars->drain), 1);
         *abort_flag = 0;
@@ -565,6 +568,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         // ---------------- epilogue: m = fma(a, G, m), v = fma(b*G, G, v) ----------------
         const int q = warp & 3;            // TMEM lane quarter this warp may read
         const int part = (warp - 2) >> 2;  // which part of the tile's columns it handles
+        const int col_split = ((int)blockDim.x / 32 - 2) / 4;  // 1 or 2 warps per lane quarter
         const uint32_t sm_g = base + G::SMEM_EPI_OFF + (uint32_t)(warp - 2) * EPI_BUF_BYTES;
         // staging buffer: 32 rows of 128 bytes; 16-byte chunk j of row r sits at (j ^ (r & 7)),
         // which makes both the row-per-thread writes and the row-segment reads conflict-free
@@ -580,7 +584,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
             const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
             const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
-            const int chunks = wi.width / (COL_SPLIT * EPI_COLS);  // chunks per warp
+            const int chunks = wi.width / (col_split * EPI_COLS);  // chunks per warp
             ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -792,15 +796,17 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
         items = tiles + rest;
     }
     const int groups = items < max_groups ? items : max_groups;
+    // 8 epilogue warps when no CTA group gets a second tile (exposed epilogue), else 4
+    const int threads = 32 * (2 + (items <= max_groups ? MAX_EPI_WARPS : 4));
     if (g_variant == 1) {
-        wgrad_fold_kernel<1><<<groups, NUM_THREADS, Geo<1>::SMEM_BYTES, p.stream>>>(
+        wgrad_fold_kernel<1><<<groups, threads, Geo<1>::SMEM_BYTES, p.stream>>>(
             map_x, map_dy, map_x3, map_dy3, map_dy3h, 0, p.m, p.v, (long long)p.ldmv, p.tokens,
             p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status);
         return cudaGetLastError();
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
-    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = Geo<2>::SMEM_BYTES;
     cfg.stream = p.stream;
     cudaLaunchAttribute attr[1];
