@@ -371,7 +371,7 @@ def run_ours(args):
 
 def load_traffic():
     """Per-launch DRAM traffic (bytes) from the committed ncu summaries, keyed by kernel; an
-    entry counts only while the kernel's source file is the one the counters were taken on."""
+    entry counts only while the kernel's source files are the ones the counters were taken on."""
     import hashlib
     p = ROOT / "profiles" / "traffic.json"
     out = {}
@@ -384,8 +384,13 @@ def load_traffic():
     for key, ent in data.items():
         if not isinstance(ent, dict):
             continue
-        src = ROOT / ent.get("source", "")
-        if src.is_file() and hashlib.sha256(src.read_bytes()).hexdigest() == ent.get("sha256"):
+        srcs = [ROOT / f for f in ent.get("sources", [])]
+        if not srcs or not all(f.is_file() for f in srcs):
+            continue
+        h = hashlib.sha256()
+        for f in srcs:
+            h.update(f.read_bytes())
+        if h.hexdigest() == ent.get("sha256"):
             out[key] = ent.get("bytes_per_launch")
     return out
 
