@@ -71,6 +71,14 @@ def load(path) -> ctypes.CDLL:
                                    ctypes.c_double, ctypes.c_double]
     L.oracle_ddp_allreduce.argtypes = [_c_double_p, _c_double_p, ctypes.c_size_t,
                                        ctypes.c_int, _c_double_p, _c_double_p]
+    L.oracle_coefficient_stats.argtypes = [_c_double_p, _c_double_p, ctypes.c_size_t,
+                                           ctypes.c_long, ctypes.c_double, _c_double_p]
+    L.oracle_sgdm_decay.argtypes = [_c_double_p, ctypes.c_size_t, ctypes.c_double]
+    L.oracle_sgdm_fold.argtypes = [_c_double_p, _c_double_p, ctypes.c_size_t, ctypes.c_int]
+    L.oracle_sgdm_update.argtypes = [_c_double_p, _c_double_p, ctypes.c_size_t, ctypes.c_double]
+    for f in (L.oracle_coefficient_stats, L.oracle_sgdm_decay, L.oracle_sgdm_fold,
+              L.oracle_sgdm_update):
+        f.restype = None
     for f in (L.oracle_decay, L.oracle_fold, L.oracle_update, L.oracle_closed_form_moments,
               L.oracle_linear_wgrad, L.oracle_linear_wgrad_entries, L.oracle_ddp_decay,
               L.oracle_ddp_allreduce):
@@ -140,6 +148,49 @@ def closed_form_moments(m, v, grads, beta1, beta2, adam_variant: bool):
     lib().oracle_closed_form_moments(_p(m), _p(v), _p(grads), n, N, beta1, beta2,
                                      1 if adam_variant else 0)
     return m, v
+
+
+def coefficient_stats(v_adama, v_adam, t: int, beta2: float) -> dict:
+    """Section 4.1: mean and range over the elements of sqrt(v_hat)/sqrt(v_hat') at step t, from
+    AdamA's second moment ``v_adama`` and standard Adam's ``v_adam`` (both as they stand after the
+    mini-batch's accumulation, before bias correction).  Elements with v_adam == 0 are left out."""
+    a = _f64(v_adama).reshape(-1)
+    b = _f64(v_adam).reshape(-1)
+    assert a.shape == b.shape
+    out = np.zeros(4)
+    lib().oracle_coefficient_stats(_p(a), _p(b), a.shape[0], int(t), float(beta2), _p(out))
+    count = int(out[3])
+    return {"sum": out[0], "min": out[1], "max": out[2], "count": count,
+            "mean": out[0] / count if count else float("nan")}
+
+
+class SGDMOracle:
+    """SGD with momentum on the same pipeline as Algorithm 2 (an extension, see the C source):
+    ``begin_minibatch`` decays the buffer by mu, ``fold`` adds grad/N, ``update`` steps."""
+
+    def __init__(self, theta, momentum=0.9):
+        self.theta = _f64(theta).reshape(-1).copy()
+        self.buf = np.zeros_like(self.theta)
+        self.mu = float(momentum)
+        self.N = None
+
+    @property
+    def n(self) -> int:
+        return self.theta.shape[0]
+
+    def begin_minibatch(self, N: int) -> None:
+        assert N >= 1
+        self.N = int(N)
+        lib().oracle_sgdm_decay(_p(self.buf), self.n, self.mu)
+
+    def fold(self, grad, lo: int = 0) -> None:
+        g = _f64(grad).reshape(-1)
+        hi = lo + g.shape[0]
+        assert 0 <= lo and hi <= self.n and self.N is not None
+        lib().oracle_sgdm_fold(_p(self.buf[lo:hi]), _p(g), g.shape[0], self.N)
+
+    def update(self, lr: float) -> None:
+        lib().oracle_sgdm_update(_p(self.theta), _p(self.buf), self.n, float(lr))
 
 
 class AdamAOracle:

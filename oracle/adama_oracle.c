@@ -13,7 +13,11 @@
  *   - Algorithm 1  : the per-mini-batch closed form of the same moments, with
  *                    standard Adam's second moment printed beside AdamA's;
  *   - Section 3.3, Eqs. 4-7 : the data-parallel variant that all-reduces the
- *                    optimizer states instead of the gradients.
+ *                    optimizer states instead of the gradients;
+ *   - Section 4.1, the figure of the coefficient sqrt(v_hat)/sqrt(v_hat'): the
+ *                    statistic that compares AdamA's adaptive scaling with Adam's;
+ *   - Discussion   : the same accumulation applied to another momentum optimizer
+ *                    (SGD with momentum).
  * Nothing is blocked, fused or reordered beyond what those passages state.
  * Loops carry an OpenMP "parallel for" over independent elements only (no
  * reduction is ever split), so results do not depend on the thread count.
@@ -190,5 +194,59 @@ ORACLE_API void oracle_ddp_allreduce(const double *m_ranks, const double *v_rank
         }
         m_out[k] = sm / (double)devices;
         v_out[k] = sv / ((double)devices * (double)devices);
+    }
+}
+
+/* Section 4.1, the coefficient between AdamA's and standard Adam's adaptive scaling at
+ * step t:  c = sqrt(v_hat) / sqrt(v_hat'),  v_hat = v/(1-beta2^t) AdamA's bias-corrected
+ * second moment and v_hat' = v'/(1-beta2^t) Adam's, both tracked over the same gradients.
+ * The paper plots, per training step, the mean of c over the elements and its range.
+ * out[0] = sum of c, out[1] = min, out[2] = max, out[3] = number of elements counted.
+ * Elements whose v' is zero have no coefficient and are left out (the paper does not say;
+ * with out[3] == 0, min is +infinity and max is 0).  Serial: one fixed summation order. */
+ORACLE_API void oracle_coefficient_stats(const double *v_adama, const double *v_adam, size_t n,
+                                         long t, double beta2, double *out) {
+    double c2 = 1.0 - pow(beta2, (double)t);
+    double sum = 0.0, lo = INFINITY, hi = 0.0, count = 0.0;
+    for (size_t k = 0; k < n; ++k) {
+        if (!(v_adam[k] > 0.0)) continue;
+        double v_hat = v_adama[k] / c2;
+        double v_hat_adam = v_adam[k] / c2;
+        double c = sqrt(v_hat) / sqrt(v_hat_adam);
+        sum += c;
+        if (c < lo) lo = c;
+        if (c > hi) hi = c;
+        count += 1.0;
+    }
+    out[0] = sum;
+    out[1] = lo;
+    out[2] = hi;
+    out[3] = count;
+}
+
+/* Extension outside the paper's algorithms (its Discussion says that other momentum
+ * optimizers can take the same accumulation): SGD with momentum mu and no dampening,
+ *     buf_t = mu*buf_{t-1} + g_t,   theta_t = theta_{t-1} - alpha*buf_t,
+ * with g_t = sum_i grad_i/N folded into buf one micro-batch at a time, as Algorithm 2
+ * folds into m.  Three steps in Algorithm 2's order: decay, fold, update. */
+ORACLE_API void oracle_sgdm_decay(double *buf, size_t n, double mu) {
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t k = 0; k < (ptrdiff_t)n; ++k) {
+        buf[k] = mu * buf[k];
+    }
+}
+
+ORACLE_API void oracle_sgdm_fold(double *buf, const double *grad, size_t n, int N) {
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t k = 0; k < (ptrdiff_t)n; ++k) {
+        double g = grad[k] / (double)N;
+        buf[k] = buf[k] + g;
+    }
+}
+
+ORACLE_API void oracle_sgdm_update(double *theta, const double *buf, size_t n, double alpha) {
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t k = 0; k < (ptrdiff_t)n; ++k) {
+        theta[k] = theta[k] - alpha * buf[k];
     }
 }

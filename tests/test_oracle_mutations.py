@@ -26,6 +26,15 @@ MUTATIONS = {
     "weight decay coupled into the gradient term": (
         "theta[k] - alpha * lambda * theta[k] - alpha * m_hat / (sqrt(v_hat) + eps)",
         "theta[k] - alpha * (m_hat + lambda * theta[k]) / (sqrt(v_hat) + eps)"),
+    "coefficient inverted": ("double c = sqrt(v_hat) / sqrt(v_hat_adam);",
+                             "double c = sqrt(v_hat_adam) / sqrt(v_hat);"),
+    "coefficient without the roots": ("double c = sqrt(v_hat) / sqrt(v_hat_adam);",
+                                      "double c = v_hat / v_hat_adam;"),
+    "coefficient counts zero v'": ("if (!(v_adam[k] > 0.0)) continue;", ""),
+    "sgdm missing 1/N": ("double g = grad[k] / (double)N;\n        buf[k]",
+                         "double g = grad[k];\n        buf[k]"),
+    "sgdm decay dropped": ("buf[k] = mu * buf[k];", "buf[k] = buf[k];"),
+    "sgdm update sign": ("theta[k] - alpha * buf[k]", "theta[k] + alpha * buf[k]"),
     "wgrad accumulates |x|": ("acc += X[(size_t)tau * ldx + (size_t)p] * dY",
                               "acc += fabs(X[(size_t)tau * ldx + (size_t)p]) * dY"),
 }
@@ -45,6 +54,11 @@ def _run_all_pins():
     pins.test_wgrad_matches_numpy_matmul()
     pins.test_wgrad_structured_inputs()
     pins.test_ddp_state_allreduce_equals_single_device_with_NR_micro_batches(2, 3)
+    pins.test_coefficient_worked_example()
+    pins.test_coefficient_for_identical_micro_gradients_is_rsqrt_n(5)
+    pins.test_coefficient_stats_bruteforce_and_bounds()
+    pins.test_sgdm_worked_example()
+    pins.test_sgdm_is_torch_sgd_on_the_mean_gradient(4)
 
 
 @pytest.mark.parametrize("name", sorted(MUTATIONS))

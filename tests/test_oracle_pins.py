@@ -12,7 +12,10 @@
   * Algorithm 1's closed form against Algorithm 2's incremental form;
   * the weight gradient against numpy's matmul and structured inputs with
     known answers;
-  * Section 3.3, Eqs. 4-7: R devices x N micro-batches == one device x N*R.
+  * Section 3.3, Eqs. 4-7: R devices x N micro-batches == one device x N*R;
+  * Section 4.1's coefficient sqrt(v_hat)/sqrt(v_hat'): hand-worked values, the 1/sqrt(N)
+    closed form for identical micro-gradients, numpy statistics, the Cauchy-Schwarz floor;
+  * the SGD-momentum extension: a hand-worked example and torch.optim.SGD in float64.
 """
 from decimal import Decimal, getcontext
 from fractions import Fraction
@@ -342,3 +345,119 @@ def test_ddp_state_allreduce_equals_single_device_with_NR_micro_batches(R, N):
             np.testing.assert_allclose(ddp.m[r], single.m, rtol=1e-12, atol=1e-20)
             np.testing.assert_allclose(ddp.v[r], single.v, rtol=1e-12)
         np.testing.assert_allclose(ddp.theta, single.theta, rtol=1e-13)
+
+
+# ----- Section 4.1 coefficient statistics and the SGD-momentum extension -----
+
+EXT_GOLDEN = Path(__file__).resolve().parent / "golden" / "extension_examples.txt"
+
+
+def _ext_rows(kind):
+    return [line.split()[1:] for line in EXT_GOLDEN.read_text().splitlines()
+            if line.startswith(kind + " ")]
+
+
+def test_coefficient_worked_example():
+    """Section 4.1's coefficient on example A, from the hand-worked v (AdamA) and v' (Adam); the
+    oracle's own two second moments on that data must give the same number."""
+    rows = [r for r in _rows() if r[0] == "A"]
+    adama = AdamAOracle([rows[0][4]], B1, B2, EPS)
+    m_adam, v_adam = np.zeros(1), np.zeros(1)
+    for (step, va, vb, c), (_, _, N, grads, *_rest) in zip(_ext_rows("COEF"), rows):
+        st = oracle.coefficient_stats([float(va)], [float(vb)], int(step), B2)
+        assert st["count"] == 1
+        for key in ("mean", "min", "max"):
+            assert st[key] == pytest.approx(float(c), rel=1e-15)
+        adama.begin_minibatch(N)
+        for g in grads:
+            adama.fold([g])
+        m_adam, v_adam = oracle.closed_form_moments(m_adam, v_adam, np.array(grads)[:, None],
+                                                    B1, B2, adam_variant=True)
+        st = oracle.coefficient_stats(adama.v, v_adam, int(step), B2)
+        assert st["mean"] == pytest.approx(float(c), rel=1e-13)
+        adama.update(LR)
+
+
+@pytest.mark.parametrize("N", [1, 2, 5])
+def test_coefficient_for_identical_micro_gradients_is_rsqrt_n(N):
+    """Identical micro-batch gradients in every mini-batch: v = v'/N at every element and step
+    (Algorithm 1's two bracket terms differ by exactly the factor N), so the coefficient is
+    1/sqrt(N) everywhere: mean = min = max; N = 1 gives exactly 1 (AdamA is Adam)."""
+    rng = np.random.default_rng(5)
+    n = 37
+    adama = AdamAOracle(np.zeros(n), B1, B2, EPS)
+    m_adam, v_adam = np.zeros(n), np.zeros(n)
+    for step in range(1, 5):
+        G = rng.normal(0, 1e-2, n)
+        adama.begin_minibatch(N)
+        for _ in range(N):
+            adama.fold(G)
+        m_adam, v_adam = oracle.closed_form_moments(m_adam, v_adam, np.tile(G, (N, 1)), B1, B2,
+                                                    adam_variant=True)
+        st = oracle.coefficient_stats(adama.v, v_adam, step, B2)
+        assert st["count"] == n
+        for key in ("mean", "min", "max"):
+            assert st[key] == pytest.approx(1.0 / np.sqrt(N), rel=1e-13)
+        adama.update(LR)
+
+
+def test_coefficient_stats_bruteforce_and_bounds():
+    """mean / min / max against numpy on independently formed arrays; zero v' elements are left
+    out; Cauchy-Schwarz keeps every coefficient at or above 1/sqrt(N)."""
+    rng = np.random.default_rng(6)
+    n, N = 50, 4
+    adama = AdamAOracle(np.zeros(n), B1, B2, EPS)
+    v_adam = np.zeros(n)
+    for step in range(1, 4):
+        grads = rng.normal(0, 1e-2, (N, n))
+        grads[:, :3] = 0.0                       # three elements never see a gradient
+        adama.begin_minibatch(N)
+        for g in grads:
+            adama.fold(g)
+        v_adam = B2 * v_adam + (1 - B2) * (grads / N).sum(0) ** 2
+        st = oracle.coefficient_stats(adama.v, v_adam, step, B2)
+        c = np.sqrt(adama.v[3:] / v_adam[3:])
+        assert st["count"] == n - 3
+        assert st["mean"] == pytest.approx(c.mean(), rel=1e-13)
+        assert st["min"] == pytest.approx(c.min(), rel=1e-13)
+        assert st["max"] == pytest.approx(c.max(), rel=1e-13)
+        assert st["min"] >= 1 / np.sqrt(N) * (1 - 1e-12)
+        assert st["max"] > 1.0 > st["min"] or N == 1
+        adama.update(LR)
+    empty = oracle.coefficient_stats(np.ones(4), np.zeros(4), 1, B2)
+    assert empty["count"] == 0 and empty["min"] == np.inf and empty["max"] == 0.0
+
+
+def test_sgdm_worked_example():
+    rows = _ext_rows("SGDM")
+    orc = oracle.SGDMOracle([float(rows[0][3])], momentum=0.9)
+    for step, N, grads, w0, buf, w1 in rows:
+        assert orc.theta[0] == pytest.approx(float(w0), rel=1e-15)
+        orc.begin_minibatch(int(N))
+        for g in grads.split(","):
+            orc.fold([float(g)])
+        assert orc.buf[0] == pytest.approx(float(buf), rel=1e-14)
+        orc.update(0.1)
+        assert orc.theta[0] == pytest.approx(float(w1), rel=1e-15)
+
+
+@pytest.mark.parametrize("N", [1, 4])
+def test_sgdm_is_torch_sgd_on_the_mean_gradient(N):
+    """The folded momentum buffer equals torch.optim.SGD's (fp64, momentum, no dampening) fed
+    with the mini-batch mean gradient, step by step."""
+    rng = np.random.default_rng(8)
+    n, mu, lr = 33, 0.8, 0.05
+    theta0 = rng.normal(0, 0.5, n)
+    orc = oracle.SGDMOracle(theta0, momentum=mu)
+    p = torch.nn.Parameter(torch.tensor(theta0, dtype=torch.float64))
+    opt = torch.optim.SGD([p], lr=lr, momentum=mu, dampening=0.0, nesterov=False, foreach=False)
+    for step in range(5):
+        grads = rng.normal(0, 1e-1, (N, n))
+        orc.begin_minibatch(N)
+        for g in grads:
+            orc.fold(g)
+        orc.update(lr)
+        p.grad = torch.tensor(grads.mean(0), dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(orc.buf, opt.state[p]["momentum_buffer"].numpy(), rtol=1e-12)
+        np.testing.assert_allclose(orc.theta, p.detach().numpy(), rtol=1e-13)
