@@ -303,6 +303,49 @@ ADAMA_API adama_status adama_linear_wgrad_fold_noalloc(
     int d_out, int64_t ldx, int64_t ldy, float *m, float *v, int64_t ldmv,
     uint32_t *status_out_host, char *err, size_t err_len, void *cuda_stream);
 
+/* ---- beside the paper's algorithms ------------------------------------------------------ */
+
+/* SGD with momentum on Algorithm 2's pipeline (the paper's Discussion remarks that other
+ * momentum optimizers can take the same accumulation; the paper gives no algorithm for it):
+ *     buf_t = mu*buf_{t-1} + sum_i grad_i/N,     w_t = w_{t-1} - lr*buf_t.
+ * adama_sgdm_fold adds one raw micro-batch gradient:  buf <- buf + grad/N  (N from
+ * adama_begin_minibatch; grad/1 under ADAMA_GRADS_PRESCALED), so no gradient buffer outlives
+ * the layer's backward step.  adama_sgdm_apply does  w <- w - lr*buf  and then stores
+ * buf <- mu*buf, the decay of the NEXT mini-batch (the same convention as adama_apply).
+ *   grad : n elements of gdt, device, read-only;  buf, w : n fp32, device, in place.
+ * 16-byte aligned pointers (8 for bf16 grad) take the 128-bit path, others a scalar one.
+ * Errors: INVALID_ARG (null pointer, dtype, lr not finite, momentum outside [0,1)), BAD_STATE
+ * (no adama_begin_minibatch yet), MISALIGNED, CUDA. */
+ADAMA_API adama_status adama_sgdm_fold(adama_ctx *ctx, const void *grad, adama_dtype gdt,
+                                       float *buf, size_t n, void *cuda_stream);
+ADAMA_API adama_status adama_sgdm_apply(adama_ctx *ctx, float *w, float *buf, size_t n, double lr,
+                                        double momentum, void *cuda_stream);
+
+/* Section 4.1, the coefficient between AdamA's and standard Adam's adaptive scaling,
+ *     c = sqrt(v_hat_t) / sqrt(v_hat_t'),
+ * v_hat AdamA's bias-corrected second moment and v_hat' the one standard Adam would hold on
+ * the same gradients (Algorithm 1, the first bracket term).  The paper plots the mean of c over
+ * the elements and its range per training step; this call produces those three numbers.
+ * Call it after the mini-batch's last fold and BEFORE adama_apply:
+ *   m, v    : the AdamA states as they stand (n fp32 each, device, read-only);
+ *   m_begin : copy of m taken right after adama_begin_minibatch, before the first fold (n fp32,
+ *             device, read-only); NULL means all zeros (the first mini-batch).  The mini-batch
+ *             gradient sum is recovered from it, (m - m_begin)/(1-beta1) = sum_i grad_i/N, so the
+ *             fused weight-gradient path needs no gradient buffer for this either;
+ *   v_adam  : Adam's second moment, n fp32, device, updated in place.  It follows the
+ *             convention of v: on entry beta2*v'_{t-1} (zeros before the first mini-batch), on
+ *             exit beta2*v'_t;
+ *   stats_dev : 4 doubles in DEVICE memory, 8-byte aligned, overwritten on the stream with
+ *             {sum of c, min c, max c, number of elements counted}; mean = sum/count.
+ * Elements whose v'_t is zero have no coefficient and are not counted; with none counted
+ * min is +infinity and max is 0.  The bias corrections of v_hat and v_hat' are equal and
+ * cancel.  Two launches (reset of stats, one pass of 20 B/element).  The sum is formed with
+ * double atomics, so its last bits may differ from run to run.
+ * Errors: INVALID_ARG, BAD_STATE (no adama_begin_minibatch yet), MISALIGNED, CUDA. */
+ADAMA_API adama_status adama_coefficient_stats(adama_ctx *ctx, const float *m, const float *m_begin,
+                                               const float *v, float *v_adam, size_t n,
+                                               double *stats_dev, void *cuda_stream);
+
 /* ---- state, checkpointing, diagnostics ------------------------------------------------- */
 
 /* Step counter t of Algorithm 2 (0 after init). */

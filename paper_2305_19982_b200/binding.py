@@ -19,7 +19,8 @@ EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
     "adama_linear_wgrad_fold", "adama_apply", "adama_apply_bf16_copy", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
-    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
+    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_sgdm_fold", "adama_sgdm_apply",
+    "adama_coefficient_stats", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
     "adama_sync_status", "adama_debug_set_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
     "adama_host_constants_allreduced", "adama_host_constants_sharded",
     "adama_version",
@@ -93,6 +94,9 @@ def load_library() -> ctypes.CDLL:
     L.adama_apply_to_host.argtypes = [vp, vp, vp, vp, sz, dbl, vp, vp]
     L.adama_linear_wgrad_fold_noalloc.argtypes = [ctypes.POINTER(_Config), ci, vp, vp, ci, ci, ci,
                                                   i64, i64, vp, vp, i64, vp, ctypes.c_char_p, sz, vp]
+    L.adama_sgdm_fold.argtypes = [vp, vp, ci, vp, sz, vp]
+    L.adama_sgdm_apply.argtypes = [vp, vp, vp, sz, dbl, dbl, vp]
+    L.adama_coefficient_stats.argtypes = [vp, vp, vp, vp, vp, sz, vp, vp]
     L.adama_get_step.argtypes = [vp]
     L.adama_get_step.restype = i64
     L.adama_set_step.argtypes = [vp, i64]
@@ -299,6 +303,52 @@ class AdamA:
             raise ValueError("w, m, v must have the same number of elements")
         self._check(self._L.adama_apply_multi(self._h, ws.ptrs, ms.ptrs, vs.ptrs, ws.ns, len(ws),
                                               float(lr), _stream_ptr(self.device)))
+
+    def sgdm_fold(self, grad: torch.Tensor, buf: torch.Tensor) -> None:
+        """adama_sgdm_fold: buf += grad/N (SGD with momentum on the same pipeline)."""
+        if not (grad.is_contiguous() and buf.is_contiguous()):
+            raise ValueError("sgdm_fold needs contiguous tensors")
+        if grad.numel() != buf.numel():
+            raise ValueError("grad and buf must have the same number of elements")
+        if grad.dtype == torch.float32:
+            gdt = F32
+        elif grad.dtype == torch.bfloat16:
+            gdt = BF16
+        else:
+            raise TypeError(f"gradient dtype {grad.dtype} not supported (float32 or bfloat16)")
+        if not grad.is_cuda:
+            raise TypeError("grad must be a CUDA tensor")
+        self._check(self._L.adama_sgdm_fold(self._h, grad.data_ptr(), gdt,
+                                            _dev_ptr(buf, torch.float32, "buf"), buf.numel(),
+                                            _stream_ptr(self.device)))
+
+    def sgdm_apply(self, w: torch.Tensor, buf: torch.Tensor, lr: float, momentum: float) -> None:
+        """adama_sgdm_apply: w -= lr*buf, then buf *= momentum for the next mini-batch."""
+        if not (w.is_contiguous() and buf.is_contiguous()):
+            raise ValueError("sgdm_apply needs contiguous tensors")
+        if w.numel() != buf.numel():
+            raise ValueError("w and buf must have the same number of elements")
+        self._check(self._L.adama_sgdm_apply(self._h, _dev_ptr(w, torch.float32, "w"),
+                                             _dev_ptr(buf, torch.float32, "buf"), w.numel(),
+                                             float(lr), float(momentum), _stream_ptr(self.device)))
+
+    def coefficient_stats(self, m: torch.Tensor, m_begin: Optional[torch.Tensor], v: torch.Tensor,
+                          v_adam: torch.Tensor, stats: torch.Tensor) -> None:
+        """adama_coefficient_stats: `stats` (4 float64 on the device) receives
+        {sum, min, max, count} of sqrt(v_hat)/sqrt(v_hat'); `v_adam` is updated in place."""
+        ts = [m, v, v_adam] + ([m_begin] if m_begin is not None else [])
+        if not all(t.is_contiguous() for t in ts):
+            raise ValueError("coefficient_stats needs contiguous tensors")
+        n = m.numel()
+        if any(t.numel() != n for t in ts):
+            raise ValueError("m, m_begin, v, v_adam must have the same number of elements")
+        if stats.numel() != 4:
+            raise ValueError("stats must hold 4 float64 values")
+        self._check(self._L.adama_coefficient_stats(
+            self._h, _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(m_begin, torch.float32, "m_begin") if m_begin is not None else None,
+            _dev_ptr(v, torch.float32, "v"), _dev_ptr(v_adam, torch.float32, "v_adam"), n,
+            _dev_ptr(stats, torch.float64, "stats"), _stream_ptr(self.device)))
 
     def apply_bf16_copy(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
                         w_bf16: torch.Tensor, lr: float) -> None:

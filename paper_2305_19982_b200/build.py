@@ -13,7 +13,8 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libadama.so"
-SOURCES = ["adama_api.cu", "fold_apply.cu", "multi_tensor.cu", "bias_grad.cu", "peer_apply.cu", "wgrad_fold.cu"]
+SOURCES = ["adama_api.cu", "fold_apply.cu", "multi_tensor.cu", "bias_grad.cu", "peer_apply.cu", "extensions.cu",
+           "wgrad_fold.cu"]
 
 
 def _nvcc() -> str:

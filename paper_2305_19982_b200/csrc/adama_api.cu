@@ -31,7 +31,7 @@ FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsig
     return c;
 }
 
-static void split_hi_lo(double x, float *hi, float *lo) {
+void split_hi_lo(double x, float *hi, float *lo) {
     *hi = (float)x;
     *lo = (float)(x - (double)*hi);
 }
@@ -514,6 +514,77 @@ adama_status adama_apply_to_host(adama_ctx *ctx, float *w, float *m, float *v, s
     cudaError_t e = cudaMemcpyAsync(w_host, w, n * sizeof(float), cudaMemcpyDeviceToHost,
                                     static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "apply_to_host copy", e);
+    return ADAMA_OK;
+}
+
+// ---- SGD with momentum on the same pipeline; coefficient statistics ----------------------------
+
+adama_status adama_sgdm_fold(adama_ctx *ctx, const void *grad, adama_dtype gdt, float *buf, size_t n,
+                             void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (gdt != ADAMA_F32 && gdt != ADAMA_BF16)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "sgdm_fold: unknown gradient dtype");
+    if (n > 0 && (!grad || !buf)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "sgdm_fold: null pointer");
+    if (ctx->n_micro < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "sgdm_fold: adama_begin_minibatch has not been called");
+    if (!aligned_to(grad, dtype_size(gdt)) || !aligned_to(buf, 4))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "sgdm_fold: pointer not aligned to its element size");
+    if (n == 0) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    const double N = (ctx->cfg.flags & ADAMA_GRADS_PRESCALED) ? 1.0 : (double)ctx->n_micro;
+    cudaError_t e = adama::launch_sgdm_fold(grad, gdt, buf, n, (float)(1.0 / N), ctx->sm_count,
+                                            static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "sgdm_fold launch", e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
+adama_status adama_sgdm_apply(adama_ctx *ctx, float *w, float *buf, size_t n, double lr,
+                              double momentum, void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (n > 0 && (!w || !buf)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "sgdm_apply: null pointer");
+    if (!isfinite(lr)) return fail(ctx, ADAMA_ERR_INVALID_ARG, "sgdm_apply: lr is not finite");
+    if (!(momentum >= 0.0) || !(momentum < 1.0))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "sgdm_apply: momentum must be in [0, 1)");
+    if (ctx->t < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE, "sgdm_apply: no mini-batch has been started (t == 0)");
+    if (!aligned_to(w, 4) || !aligned_to(buf, 4))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "sgdm_apply: pointer not aligned to 4 bytes");
+    if (n == 0) return ADAMA_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    float mu_hi, mu_lo;
+    adama::split_hi_lo(momentum, &mu_hi, &mu_lo);
+    cudaError_t e = adama::launch_sgdm_apply(w, buf, n, (float)lr, mu_hi, mu_lo, ctx->sm_count,
+                                             static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "sgdm_apply launch", e);
+    ctx->launches += 1;
+    return ADAMA_OK;
+}
+
+adama_status adama_coefficient_stats(adama_ctx *ctx, const float *m, const float *m_begin,
+                                     const float *v, float *v_adam, size_t n, double *stats_dev,
+                                     void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (!stats_dev || (n > 0 && (!m || !v || !v_adam)))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "coefficient_stats: null pointer");
+    if (ctx->n_micro < 1)
+        return fail(ctx, ADAMA_ERR_BAD_STATE,
+                    "coefficient_stats: adama_begin_minibatch has not been called");
+    if (!(ctx->cfg.beta1 < 1.0))
+        return fail(ctx, ADAMA_ERR_UNSUPPORTED, "coefficient_stats: needs beta1 < 1");
+    if (!aligned_to(m, 4) || !aligned_to(v, 4) || !aligned_to(v_adam, 4) ||
+        (m_begin && !aligned_to(m_begin, 4)) || !aligned_to(stats_dev, 8))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "coefficient_stats: pointer not aligned");
+    DeviceGuard guard(ctx->cfg.device);
+    adama::CoefConstants c;
+    const double om1 = 1.0 - ctx->cfg.beta1;
+    c.k = (float)((1.0 - ctx->cfg.beta2) / (om1 * om1));
+    adama::split_hi_lo(ctx->cfg.beta2, &c.beta2_hi, &c.beta2_lo);
+    cudaError_t e = adama::launch_coefficient_stats(m, m_begin, v, v_adam, n, c, stats_dev,
+                                                    ctx->sm_count,
+                                                    static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "coefficient_stats launch", e);
+    ctx->launches += (n > 0 ? 2 : 1);
     return ADAMA_OK;
 }
 

@@ -28,6 +28,17 @@ struct ApplyConstants {
     float w_keep;    // 1 - lr*weight_decay (decoupled decay, AdamW); exactly 1 when it is off
 };
 
+// Coefficient statistics (Section 4.1): k = (1-beta2)/(1-beta1)^2 turns the squared change of m
+// over a mini-batch into Adam's second-moment increment; beta2 = hi + lo as in ApplyConstants.
+struct CoefConstants {
+    float k;
+    float beta2_hi;
+    float beta2_lo;
+};
+
+// x = hi + lo with hi = fp32(x)
+void split_hi_lo(double x, float *hi, float *lo);
+
 FoldConstants make_fold_constants(double beta1, double beta2, int n_micro, unsigned flags);
 // world > 1: m and v hold the SUM over `world` data-parallel ranks (Section 3.3 of the paper);
 // the 1/world and 1/world^2 of Eqs. 6-7 and the world*beta2 pre-scaling of the next mini-batch
@@ -48,6 +59,16 @@ cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, s
 // w_bf16_out (may be null): n bf16 elements that receive the updated weights, rounded to nearest
 cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants c, int sm_count,
                          cudaStream_t stream, void *w_bf16_out = nullptr);
+
+// SGD-momentum fold / apply and the coefficient statistics (extensions.cu)
+cudaError_t launch_sgdm_fold(const void *grad, adama_dtype gdt, float *buf, size_t n, float inv_n,
+                             int sm_count, cudaStream_t stream);
+cudaError_t launch_sgdm_apply(float *w, float *buf, size_t n, float lr, float mu_hi, float mu_lo,
+                              int sm_count, cudaStream_t stream);
+// stats: 4 doubles in device memory {sum, min, max, count}; two launches (reset, pass)
+cudaError_t launch_coefficient_stats(const float *m, const float *m_begin, const float *v,
+                                     float *v_adam, size_t n, CoefConstants c, double *stats,
+                                     int sm_count, cudaStream_t stream);
 
 // multi-tensor forms (multi_tensor.cu): up to kMultiMax tensors per launch, each shorter than
 // 2^32 * 4096 elements in total blocks

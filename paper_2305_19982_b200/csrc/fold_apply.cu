@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 
 #include "adama_device.cuh"
+#include "stream_access.cuh"
 
 namespace adama {
 namespace {
@@ -32,57 +33,6 @@ namespace {
 constexpr int kThreads = ADAMA_STREAM_THREADS;
 constexpr int kCtasPerSm = ADAMA_FOLD_CTAS_PER_SM;        // fold: 6 x (g, m, v) vectors in flight per thread
 constexpr int kApplyCtasPerSm = ADAMA_APPLY_CTAS_PER_SM;  // apply: 8 x (w, m, v) vectors = 96 data registers
-
-// ---- 128-bit global accesses ------------------------------------------------------------
-// m, v and w are read once and written once per pass, the gradient is read once:
-// loads do not allocate in L1.
-__device__ __forceinline__ float4 ld_stream(const float4 *p) {
-    float4 r;
-    asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
-                 : "l"(p));
-    return r;
-}
-__device__ __forceinline__ uint2 ld_stream_ro(const uint2 *p) {
-    uint2 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
-    return r;
-}
-__device__ __forceinline__ float4 ld_stream_ro(const float4 *p) {
-    float4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
-                 : "l"(p));
-    return r;
-}
-__device__ __forceinline__ void st_stream(float4 *p, float4 x) {
-#ifdef ADAMA_ST_CS
-    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z),
-                 "f"(x.w)
-                 : "memory");
-    return;
-#endif
-    asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z),
-                 "f"(x.w)
-                 : "memory");
-}
-
-// four gradient values widened exactly to fp32
-struct Grad4 {
-    float x, y, z, w;
-};
-__device__ __forceinline__ Grad4 load_grad4(const float *g, size_t i4) {
-    float4 t = ld_stream_ro(reinterpret_cast<const float4 *>(g) + i4);
-    return {t.x, t.y, t.z, t.w};
-}
-__device__ __forceinline__ Grad4 load_grad4(const __nv_bfloat16 *g, size_t i4) {
-    uint2 t = ld_stream_ro(reinterpret_cast<const uint2 *>(g) + i4);
-    // bf16 -> fp32 is a 16-bit left shift
-    return {__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
-            __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u)};
-}
-__device__ __forceinline__ float widen(float g) { return g; }
-__device__ __forceinline__ float widen(__nv_bfloat16 g) { return __bfloat162float(g); }
 
 template <typename G, int UNROLL>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
@@ -210,17 +160,6 @@ apply_scalar_kernel(float *__restrict__ w, float *__restrict__ m, float *__restr
     }
 }
 
-inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-
-// Grid: enough CTAs to cover the data once, capped at a whole number of CTAs per SM.
-inline unsigned grid_for(size_t work_items, size_t items_per_cta, int sm_count,
-                         int ctas_per_sm = kCtasPerSm) {
-    size_t need = (work_items + items_per_cta - 1) / items_per_cta;
-    size_t cap = (size_t)sm_count * ctas_per_sm;
-    if (need < 1) need = 1;
-    return (unsigned)(need < cap ? need : cap);
-}
-
 }  // namespace
 
 cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, size_t n,
@@ -232,20 +171,20 @@ cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, s
     if (gdt == ADAMA_F32) {
         const float *g = static_cast<const float *>(grad);
         if (vec) {
-            unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count);
+            unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count, kCtasPerSm);
             fold_vec_kernel<float, U><<<grid, kThreads, 0, stream>>>(g, m, v, n4, n, c.a, c.b);
         } else {
-            unsigned grid = grid_for(n, kThreads, sm_count);
+            unsigned grid = grid_for(n, kThreads, sm_count, kCtasPerSm);
             fold_scalar_kernel<float><<<grid, kThreads, 0, stream>>>(g, m, v, n, c.a, c.b);
         }
     } else {
         const __nv_bfloat16 *g = static_cast<const __nv_bfloat16 *>(grad);
         if (vec) {
-            unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count);
+            unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count, kCtasPerSm);
             fold_vec_kernel<__nv_bfloat16, U><<<grid, kThreads, 0, stream>>>(g, m, v, n4, n, c.a,
                                                                               c.b);
         } else {
-            unsigned grid = grid_for(n, kThreads, sm_count);
+            unsigned grid = grid_for(n, kThreads, sm_count, kCtasPerSm);
             fold_scalar_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>(g, m, v, n, c.a, c.b);
         }
     }
@@ -265,7 +204,7 @@ cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants 
         else
             apply_vec_kernel<U, false><<<grid, kThreads, 0, stream>>>(w, m, v, nullptr, n4, n, c);
     } else {
-        unsigned grid = grid_for(n, kThreads, sm_count);
+        unsigned grid = grid_for(n, kThreads, sm_count, kCtasPerSm);
         apply_scalar_kernel<<<grid, kThreads, 0, stream>>>(w, m, v, wb, n, c);
     }
     return cudaGetLastError();
