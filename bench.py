@@ -2,7 +2,7 @@
 """Benchmark of the AdamA hot path on B200: fold / apply GB/s and fused wgrad+fold TFLOP/s.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors]
+                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors|extensions]
 
 One step of the headline workload = one pass of the whole path:
   phase A  (flat 335M-parameter buffer, bf16 gradients, N=8):
@@ -625,6 +625,53 @@ def run_sweep(args):
     opt.close()
 
 
+def run_extensions(args):
+    """The kernels beside the headline path at the flat workload's size (335 M elements, inputs far
+    above the L2): SGD-momentum fold / apply, the coefficient statistics, apply with the bf16
+    copy.  Median of 20 launches each, CUDA events, against the same HBM peak."""
+    import paper_2305_19982_b200 as adama
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pk = peaks()
+    n = wl.CONFIG2_FULL_N
+    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
+    opt.begin_minibatch(wl.CONFIG2.n_micro)
+    w = wl.normal((n,), 0.02, torch.float32, 1, device=dev)
+    m = wl.normal((n,), 1e-4, torch.float32, 3, device=dev)
+    m0 = wl.normal((n,), 1e-4, torch.float32, 4, device=dev)
+    v = wl.normal((n,), 1e-4, torch.float32, 5, device=dev).square_()
+    va = v.clone()
+    g = wl.normal((n,), wl.CONFIG2.grad_std, torch.bfloat16, 2, device=dev)
+    wb = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    stats = torch.zeros(4, dtype=torch.float64, device=dev)
+    rows = {}
+    for name, call, bpp in (
+            ("sgdm_fold_bf16", lambda: opt.sgdm_fold(g, m), 2 + 8),
+            ("sgdm_apply", lambda: opt.sgdm_apply(w, m, 1e-3, 0.9), 16),
+            ("coefficient_stats", lambda: opt.coefficient_stats(m, m0, v, va, stats), 20),
+            ("apply_bf16_copy", lambda: opt.apply_bf16_copy(w, m, v, wb, wl.LR), 26)):
+        for _ in range(3):
+            call()
+        ts = []
+        for _ in range(20):
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ts.sort()
+        med = ts[len(ts) // 2]
+        rows[name] = {"ms_median": med, "ms_best": ts[0], "bytes_per_param": bpp,
+                      "GBps_median": bpp * n / (med * 1e-3) / 1e9,
+                      "frac_of_peak": bpp * n / (med * 1e-3) / 1e9 / pk["hbm_gbs"]}
+    print(json.dumps({"metric": "adama_extension_kernels", "unit": "GB/s", "params": n,
+                      "peak": pk["hbm_gbs"], "peak_source": pk["source"],
+                      "l2": "inputs larger than L2, no flush", "rows": rows}), flush=True)
+    opt.close()
+
+
 def run_small_tensors(args):
     """The non-matrix parameters of a GPT-2-XL-shaped model (per block: two norms, four biases;
     432 tensors, 1.0 M elements): one mini-batch of N=8 folds + apply with the multi-tensor
@@ -686,7 +733,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
-    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors"])
+    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -695,6 +742,8 @@ def main():
         run_reference(args)
     elif args.workload == "sweep":
         run_sweep(args)
+    elif args.workload == "extensions":
+        run_extensions(args)
     elif args.workload == "small_tensors":
         args.steps = min(args.steps, 10)
         run_small_tensors(args)
