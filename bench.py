@@ -2,7 +2,7 @@
 """Benchmark of the AdamA hot path on B200: fold / apply GB/s and fused wgrad+fold TFLOP/s.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors|extensions]
+                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors|extensions|oracle_timing]
 
 One step of the headline workload = one pass of the whole path:
   phase A  (flat 335M-parameter buffer, bf16 gradients, N=8):
@@ -672,6 +672,61 @@ def run_extensions(args):
     opt.close()
 
 
+def run_oracle_timing(args):
+    """The oracle's own kernels timed on the host cores, with 1 thread and with all of them: fold
+    and update at 2^20 and 2^24 elements (M params/s and effective GB/s at 18 and 24 B/param, the
+    GPU kernels' byte counts), the naive weight gradient at 1024^3 (GFLOP/s).  A baseline beside
+    the GPU numbers, nothing more; the oracle is timed as it stands."""
+    import platform
+
+    import numpy as np
+
+    import oracle
+    all_threads = oracle.num_threads()
+    rows = []
+    rng = np.random.default_rng(0)
+    for threads in sorted({1, all_threads}):
+        oracle.set_num_threads(threads)
+        for n in (1 << 20, 1 << 24):
+            orc = oracle.AdamAOracle(rng.normal(0, 0.02, n), wl.BETA1, wl.BETA2, wl.EPS)
+            g = rng.normal(0, 1e-3, n)
+            orc.begin_minibatch(8)
+            reps = 20 if n <= (1 << 20) else 3
+            orc.fold(g)
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                orc.fold(g)
+            tf = (time.perf_counter() - t0) / reps
+            orc.update(wl.LR)
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                orc.update(wl.LR)
+            tu = (time.perf_counter() - t0) / reps
+            rows.append({"threads": threads, "n": n,
+                         "fold_Mparams_per_s": n / tf / 1e6, "fold_GBps_at_18B": 18 * n / tf / 1e9,
+                         "update_Mparams_per_s": n / tu / 1e6,
+                         "update_GBps_at_24B": 24 * n / tu / 1e9})
+        d = 1024
+        X = rng.normal(0, 1, (d, d))
+        dY = rng.normal(0, 1e-2, (d, d))
+        t0 = time.perf_counter()
+        oracle.linear_wgrad(X, dY)
+        tg = time.perf_counter() - t0
+        rows.append({"threads": threads, "wgrad": "1024^3", "seconds": tg,
+                     "GFLOPps": 2.0 * d ** 3 / tg / 1e9})
+    oracle.set_num_threads(all_threads)
+    cpu = platform.processor() or platform.machine()
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.startswith("model name"):
+                cpu = ln.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    print(json.dumps({"metric": "adama_oracle_host_timing", "kind": "oracle", "cores": all_threads,
+                      "cpu": cpu, "rows": rows}), flush=True)
+
+
 def run_small_tensors(args):
     """The non-matrix parameters of a GPT-2-XL-shaped model (per block: two norms, four biases;
     432 tensors, 1.0 M elements): one mini-batch of N=8 folds + apply with the multi-tensor
@@ -733,7 +788,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
-    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions"])
+    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -744,6 +799,8 @@ def main():
         run_sweep(args)
     elif args.workload == "extensions":
         run_extensions(args)
+    elif args.workload == "oracle_timing":
+        run_oracle_timing(args)
     elif args.workload == "small_tensors":
         args.steps = min(args.steps, 10)
         run_small_tensors(args)

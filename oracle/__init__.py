@@ -46,6 +46,8 @@ def load(path) -> ctypes.CDLL:
     """dlopen one build of the oracle and declare its signatures."""
     L = ctypes.CDLL(str(path))
     L.oracle_num_threads.restype = ctypes.c_int
+    L.oracle_set_num_threads.argtypes = [ctypes.c_int]
+    L.oracle_set_num_threads.restype = None
     L.oracle_decay.argtypes = [_c_double_p, _c_double_p, ctypes.c_size_t,
                                ctypes.c_double, ctypes.c_double]
     L.oracle_fold.argtypes = [_c_double_p, _c_double_p, _c_double_p, ctypes.c_size_t,
@@ -95,6 +97,11 @@ def lib() -> ctypes.CDLL:
 
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
+
+
+def set_num_threads(threads: int) -> None:
+    """Thread count of the oracle's loops from now on (timing only; results do not change)."""
+    lib().oracle_set_num_threads(int(threads))
 
 
 def _f64(a) -> np.ndarray:

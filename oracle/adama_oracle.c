@@ -49,6 +49,16 @@ ORACLE_API int oracle_num_threads(void) {
 #endif
 }
 
+/* Limits the threads of the loops below (timing with 1 thread and with all cores); no
+ * effect on results, since no reduction is split across threads. */
+ORACLE_API void oracle_set_num_threads(int threads) {
+#ifdef _OPENMP
+    if (threads >= 1) omp_set_num_threads(threads);
+#else
+    (void)threads;
+#endif
+}
+
 /* Algorithm 2, first line of the while-body: m_t <- beta1*m_{t-1},
  * v_t <- beta2*v_{t-1}.  (The step counter t <- t+1 is kept by the caller.) */
 ORACLE_API void oracle_decay(double *m, double *v, size_t n, double beta1, double beta2) {
