@@ -170,6 +170,44 @@ def test_full_size_config2_sampled():
     opt.close()
 
 
+def test_more_than_2_to_32_elements_sampled():
+    """n = 2^32 + 7: element indices and byte offsets beyond 32 bits (the largest size the
+    workloads reach is 335 M; this is the index-arithmetic edge).  One mini-batch with N = 2;
+    head, tail and windows around 2^31 and 2^32 are checked element by element."""
+    n = (1 << 32) + 7
+    win = torch.arange(-2050, 2050)
+    idx = torch.cat([torch.arange(0, 4096), (1 << 31) + win, (1 << 32) + win[win < 7],
+                     torch.arange(0, n, 1_000_003)]).unique()
+    idx = idx[(idx >= 0) & (idx < n)]
+    idx_d = idx.cuda()
+    opt = adama.AdamA()
+    w = wl.normal((n,), 0.02, torch.float32, wl.seed_for(9, 99), device="cuda")
+    m = torch.zeros(n, device="cuda")
+    v = torch.zeros(n, device="cuda")
+    orc = AdamAOracle(f64(w[idx_d]))
+    opt.begin_minibatch(2)
+    orc.begin_minibatch(2)
+    for i in range(2):
+        g = wl.normal((n,), 1e-3, torch.bfloat16, wl.seed_for(9, 0, i), device="cuda")
+        opt.fold(g, m, v)
+        orc.fold(f64(g[idx_d]))
+        del g
+    assert rel_l2(f64(m[idx_d]), orc.m) <= TOL
+    assert rel_l2(f64(v[idx_d]), orc.v) <= TOL
+    opt.apply(w, m, v, wl.LR)
+    orc.update(wl.LR)
+    assert rel_l2(f64(w[idx_d]), orc.theta) <= TOL
+    assert rel_l2(f64(m[idx_d]), wl.BETA1 * orc.m) <= TOL
+    assert rel_l2(f64(v[idx_d]), wl.BETA2 * orc.v) <= TOL
+    # every element was visited exactly once: with two N(0, 1e-3) gradients v > 0 almost surely,
+    # and a second visit would show as a second decay
+    assert int((v == 0).sum()) < 1000
+    opt.sync_status()
+    opt.close()
+    del w, m, v
+    torch.cuda.empty_cache()
+
+
 def test_decoupled_weight_decay_extension():
     """adama_set_weight_decay (AdamW-style, beyond the paper's algorithms) against the oracle's
     pinned decoupled-decay update; and lambda = 0 stays bit-identical to the plain update."""

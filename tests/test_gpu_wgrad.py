@@ -190,6 +190,13 @@ def test_config5_layer_shapes_sampled(name, d_in, d_out):
     _sampled_parity(wl.CONFIG5_TOKENS, d_in, d_out, 1, 1, 5, count=1500)
 
 
+def test_weight_matrix_beyond_2_to_31_elements_sampled():
+    """49152 x 49152 weights (2.4 G elements: element offsets into m, v beyond 31 bits, byte
+    offsets beyond 33), 64 tokens: sampled entries plus the bottom-right tile."""
+    _sampled_parity(64, 49152, 49152, 1, 1, 10, count=4000)
+    torch.cuda.empty_cache()
+
+
 def test_zero_tokens_is_a_noop():
     opt = adama.AdamA()
     opt.begin_minibatch(1)
