@@ -142,6 +142,22 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
                                                int64_t ldy, float *m, float *v, int64_t ldmv,
                                                void *cuda_stream);
 
+/* adama_linear_wgrad_fold that also folds the layer's bias gradient, the column sums of dY,
+ *     g[q] = sum_{tau < tokens} dY[tau,q],   m_bias[q] += a*g[q],   v_bias[q] += b*g[q]^2
+ * (Algorithm 2, inner loop body, for the bias of the same layer) in the same launch: the
+ * kernel's epilogue warps, idle until the first accumulator tile is complete, form the sums
+ * meanwhile; every 32-column slab is summed over all tokens by one CTA, so the sum is
+ * complete before it is squared, and the result is deterministic.
+ *   m_bias, v_bias : d_out fp32 elements each, contiguous, device, updated in place.
+ * Weight results are bit-identical to adama_linear_wgrad_fold; the bias results equal
+ * adama_bias_grad_fold's up to the order of the fp32 token sum.
+ * Errors: as adama_linear_wgrad_fold, plus INVALID_ARG (null bias moments), MISALIGNED. */
+ADAMA_API adama_status adama_linear_wgrad_bias_fold(adama_ctx *ctx, const void *X, const void *dY,
+                                                    int tokens, int d_in, int d_out, int64_t ldx,
+                                                    int64_t ldy, float *m, float *v, int64_t ldmv,
+                                                    float *m_bias, float *v_bias,
+                                                    void *cuda_stream);
+
 /* Algorithm 2, "Update", fused with the first line of the NEXT loop body:
  *     m_hat = m/(1-beta1^t), v_hat = v/(1-beta2^t),
  *     w <- w - lr * m_hat / (sqrt(v_hat) + eps)

@@ -17,7 +17,7 @@ _LIB_PATH = _PKG / "libadama.so"
 
 EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
-    "adama_linear_wgrad_fold", "adama_apply", "adama_apply_bf16_copy", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
+    "adama_linear_wgrad_fold", "adama_linear_wgrad_bias_fold", "adama_apply", "adama_apply_bf16_copy", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_sgdm_fold", "adama_sgdm_apply",
     "adama_coefficient_stats", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
@@ -75,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     L.adama_begin_minibatch.argtypes = [vp, ci]
     L.adama_fold.argtypes = [vp, vp, ci, vp, vp, sz, vp]
     L.adama_linear_wgrad_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp]
+    L.adama_linear_wgrad_bias_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp, vp, vp]
     L.adama_apply.argtypes = [vp, vp, vp, vp, sz, dbl, vp]
     L.adama_apply_bf16_copy.argtypes = [vp, vp, vp, vp, vp, sz, dbl, vp]
     L.adama_apply_allreduced.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
@@ -215,9 +216,12 @@ class AdamA:
                                        _stream_ptr(self.device)))
 
     def linear_wgrad_fold(self, X: torch.Tensor, dY: torch.Tensor, m: torch.Tensor,
-                          v: torch.Tensor) -> None:
+                          v: torch.Tensor, m_bias: Optional[torch.Tensor] = None,
+                          v_bias: Optional[torch.Tensor] = None) -> None:
         """adama_linear_wgrad_fold: X [tokens, d_in], dY [tokens, d_out] bf16 (unit stride in
-        the last dim), m, v [d_in, d_out] fp32 views with a common row pitch."""
+        the last dim), m, v [d_in, d_out] fp32 views with a common row pitch.  With m_bias and
+        v_bias (contiguous, d_out fp32 each): adama_linear_wgrad_bias_fold, which folds the
+        bias gradient (column sums of dY) in the same launch."""
         if X.dim() != 2 or dY.dim() != 2 or m.dim() != 2 or v.dim() != 2:
             raise ValueError("linear_wgrad_fold takes 2-D tensors")
         tokens, d_in = X.shape
@@ -234,6 +238,18 @@ class AdamA:
         ldx = X.stride(0) if tokens > 1 else max(d_in, X.stride(0))
         ldy = dY.stride(0) if tokens > 1 else max(d_out, dY.stride(0))
         ldmv = m.stride(0) if d_in > 1 else max(d_out, m.stride(0))
+        if (m_bias is None) != (v_bias is None):
+            raise ValueError("m_bias and v_bias go together")
+        if m_bias is not None:
+            if m_bias.numel() != d_out or v_bias.numel() != d_out or not (
+                    m_bias.is_contiguous() and v_bias.is_contiguous()):
+                raise ValueError("m_bias, v_bias must be contiguous with d_out elements")
+            self._check(self._L.adama_linear_wgrad_bias_fold(
+                self._h, _dev_ptr(X, torch.bfloat16, "X"), _dev_ptr(dY, torch.bfloat16, "dY"),
+                tokens, d_in, d_out, ldx, ldy, _dev_ptr(m, torch.float32, "m"),
+                _dev_ptr(v, torch.float32, "v"), ldmv, _dev_ptr(m_bias, torch.float32, "m_bias"),
+                _dev_ptr(v_bias, torch.float32, "v_bias"), _stream_ptr(self.device)))
+            return
         self._check(self._L.adama_linear_wgrad_fold(
             self._h, _dev_ptr(X, torch.bfloat16, "X"), _dev_ptr(dY, torch.bfloat16, "dY"),
             tokens, d_in, d_out, ldx, ldy, _dev_ptr(m, torch.float32, "m"),

@@ -218,9 +218,9 @@ adama_status adama_fold(adama_ctx *ctx, const void *grad, adama_dtype gdt, float
     return ADAMA_OK;
 }
 
-adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *dY, int tokens,
-                                     int d_in, int d_out, int64_t ldx, int64_t ldy, float *m,
-                                     float *v, int64_t ldmv, void *cuda_stream) {
+static adama_status wgrad_impl(adama_ctx *ctx, const void *X, const void *dY, int tokens, int d_in,
+                               int d_out, int64_t ldx, int64_t ldy, float *m, float *v,
+                               int64_t ldmv, float *bias_m, float *bias_v, void *cuda_stream) {
     adama_status st = check_wgrad_args(ctx, X, dY, tokens, d_in, d_out, ldx, ldy, m, v, ldmv);
     if (st != ADAMA_OK) return st;
     if (tokens == 0) return ADAMA_OK;  // empty sum: G = 0, nothing to add
@@ -240,11 +240,33 @@ adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *
     a.status = ctx->status_dev;
     a.sm_count = ctx->sm_count;
     a.stream = static_cast<cudaStream_t>(cuda_stream);
+    a.bias_m = bias_m;
+    a.bias_v = bias_v;
     const char *msg = "wgrad_fold";
     cudaError_t e = adama::launch_wgrad_fold(a, &msg);
     if (e != cudaSuccess) return cuda_fail(ctx, msg, e);
     ctx->launches += 1;
     return ADAMA_OK;
+}
+
+adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, const void *dY, int tokens,
+                                     int d_in, int d_out, int64_t ldx, int64_t ldy, float *m,
+                                     float *v, int64_t ldmv, void *cuda_stream) {
+    return wgrad_impl(ctx, X, dY, tokens, d_in, d_out, ldx, ldy, m, v, ldmv, nullptr, nullptr,
+                      cuda_stream);
+}
+
+adama_status adama_linear_wgrad_bias_fold(adama_ctx *ctx, const void *X, const void *dY, int tokens,
+                                          int d_in, int d_out, int64_t ldx, int64_t ldy, float *m,
+                                          float *v, int64_t ldmv, float *m_bias, float *v_bias,
+                                          void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (!m_bias || !v_bias)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_bias_fold: null bias moments");
+    if (!aligned_to(m_bias, 4) || !aligned_to(v_bias, 4))
+        return fail(ctx, ADAMA_ERR_MISALIGNED, "wgrad_bias_fold: bias moments not aligned to 4 bytes");
+    return wgrad_impl(ctx, X, dY, tokens, d_in, d_out, ldx, ldy, m, v, ldmv, m_bias, v_bias,
+                      cuda_stream);
 }
 
 static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,

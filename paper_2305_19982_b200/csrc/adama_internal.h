@@ -101,6 +101,10 @@ struct WgradArgs {
     unsigned *status;  // device status block
     int sm_count;
     cudaStream_t stream;
+    // optional: moments of the layer's bias (d_out fp32 each); the column sums of dY are
+    // folded into them by the same launch
+    float *bias_m = nullptr;
+    float *bias_v = nullptr;
 };
 // Returns cudaSuccess or the failing CUDA error; *msg (static string) says which step failed.
 cudaError_t launch_wgrad_fold(const WgradArgs &args, const char **msg);

@@ -41,6 +41,7 @@
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the kernel
 // records a code in the status block, all roles drain and leave, TMEM is freed.
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include <cstdlib>
 
@@ -70,11 +71,17 @@ constexpr int EPI_BUF_BYTES = EPI_ROWS * EPI_COLS * 4;  // 4096: one transpositi
 // (1600x1600: 41.8 vs 43.8 us).
 constexpr int MAX_EPI_WARPS = 8;
 constexpr int EPI_BYTES = MAX_EPI_WARPS * EPI_BUF_BYTES;
-constexpr int MAX_THREADS = 32 * (2 + MAX_EPI_WARPS);
+constexpr int MAX_THREADS = 32 * (2 + MAX_EPI_WARPS + 2);  // + the two optional bias warps
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
 constexpr int MAX_STAGES = 12;
 constexpr int SMEM_BAR_BYTES = 256;
+#ifndef ADAMA_WGRAD_BIAS_UNROLL
+#define ADAMA_WGRAD_BIAS_UNROLL 8
+#endif
+constexpr int BIAS_UNROLL = ADAMA_WGRAD_BIAS_UNROLL;  // 16-byte loads in flight per thread of a bias warp
+constexpr int BIAS_WARPS = 2;
+constexpr int SMEM_BIAS_BYTES = BIAS_WARPS * 32 * 4;
 
 // Per-variant geometry: CTAS = CTAs cooperating on one tile (1 or 2).
 template <int CTAS>
@@ -90,7 +97,8 @@ struct Geo {
     static constexpr int STAGES = CTAS == 1 ? 4 * 64 / BK : ADAMA_WGRAD_STAGES;
     static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
-    static constexpr int SMEM_BYTES = SMEM_BAR_OFF + SMEM_BAR_BYTES + 1024;  // + alignment slack
+    static constexpr int SMEM_BIAS_OFF = SMEM_BAR_OFF + SMEM_BAR_BYTES;
+    static constexpr int SMEM_BYTES = SMEM_BIAS_OFF + SMEM_BIAS_BYTES + 1024;  // + alignment slack
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(STAGES <= MAX_STAGES, "barrier block");
     // tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both
@@ -306,6 +314,15 @@ __device__ __forceinline__ float4 ld_global_v4_stream(const float *p) {
                  : "l"(p));
     return r;
 }
+// read-only data that this SM reads once: no L1 allocation (the L1 left beside 200+ KB of
+// shared memory is small and serves the epilogue)
+__device__ __forceinline__ uint4 ld_global_nc_v4(const void *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
 __device__ __forceinline__ void st_global_v4(float *p, float4 x) {
     asm volatile("st.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z),
                  "f"(x.w)
@@ -382,7 +399,9 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   const __grid_constant__ CUtensorMap map_dy3h, int grouped,
                   float *__restrict__ m_out,
                   float *__restrict__ v_out, long long ldmv, int tokens, int d_in, int d_out,
-                  int split_from, int num_items, float a, float b, unsigned *status) {
+                  int split_from, int num_items, float a, float b, unsigned *status,
+                  const __nv_bfloat16 *__restrict__ dy_raw, long long ldy,
+                  float *__restrict__ bias_m, float *__restrict__ bias_v) {
     using G = Geo<CTAS>;
     constexpr int STAGES = G::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -399,6 +418,8 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     const int num_groups = gridDim.x / CTAS;
     const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
     const int num_kb = (tokens + BK - 1) / BK;
+    // warps 2 .. 2+epi_warps-1: epilogue; with bias moments, BIAS_WARPS more after them
+    const int epi_warps = (int)blockDim.x / 32 - 2 - (bias_m != nullptr ? BIAS_WARPS : 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -407,7 +428,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         }
         for (int s = 0; s < ACC_STAGES; ++s) {
             mbar_init(smem_u32(&bars->acc_full[s]), 1);
-            mbar_init(smem_u32(&bars->acc_empty[s]), (blockDim.x / 32 - 2) * CTAS);
+            mbar_init(smem_u32(&bars->acc_empty[s]), epi_warps * CTAS);
         }
         mbar_init(smem_u32(&bars->drain), 1);
         *abort_flag = 0;
@@ -564,11 +585,90 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             }
         }
         __syncwarp();
+    } else if (warp >= 2 + epi_warps) {
+        // ---------------- bias gradient: column sums of dY, folded into the bias moments ----------------
+        // Two extra warps (present only when bias moments were passed) work through the layer's
+        // bias gradient while the other roles run the tiles, straight from global memory (the
+        // producer pulls the same dY through the L2 anyway).  A CTA takes whole 32-column slabs
+        // over ALL tokens, so a token sum is complete before it is squared and no CTA depends
+        // on another: a warp load covers 8 rows x 64 bytes, 8 loads in flight per thread (4 make these
+        // warps the last to finish on wide layers, 16 take more from the main loop's loads), sums
+        // combined across the 8 row lanes by shuffles and across the two warps through shared
+        // memory, in fixed order.  These warps wait on no mbarrier, so the named barrier
+        // between them cannot be left waiting by a role that gave up.
+        const int ew = warp - (2 + epi_warps);
+        const int slabs = (d_out + 31) / 32;
+        float *red = reinterpret_cast<float *>(smem + G::SMEM_BIAS_OFF);  // [BIAS_WARPS][32]
+        const int rsub = lane >> 2;  // row within a group of 8
+        const int cq = lane & 3;     // 16-byte chunk of the slab's 64-byte row segment
+        const int step = BIAS_WARPS * 8;
+        for (int slab = (int)blockIdx.x; slab < slabs; slab += (int)gridDim.x) {
+            const int col = slab * 32 + cq * 8;
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            if (col + 8 <= d_out) {
+                const __nv_bfloat16 *src = dy_raw + col;
+                int tau = ew * 8 + rsub;
+                for (; tau + (BIAS_UNROLL - 1) * step < tokens; tau += BIAS_UNROLL * step) {
+                    uint4 x[BIAS_UNROLL];
+#pragma unroll
+                    for (int u = 0; u < BIAS_UNROLL; ++u)
+                        x[u] = ld_global_nc_v4(src + (long long)(tau + u * step) * ldy);
+#pragma unroll
+                    for (int u = 0; u < BIAS_UNROLL; ++u) {
+                        const unsigned wds[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            acc[2 * k] += __uint_as_float(wds[k] << 16);
+                            acc[2 * k + 1] += __uint_as_float(wds[k] & 0xffff0000u);
+                        }
+                    }
+                }
+                for (; tau < tokens; tau += step) {
+                    const uint4 x = ld_global_nc_v4(src + (long long)tau * ldy);
+                    const unsigned wds[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        acc[2 * k] += __uint_as_float(wds[k] << 16);
+                        acc[2 * k + 1] += __uint_as_float(wds[k] & 0xffff0000u);
+                    }
+                }
+            } else {
+                // ragged last columns: element-wise, bounds-checked
+                for (int tau = ew * 8 + rsub; tau < tokens; tau += step)
+                    for (int e = 0; e < 8; ++e)
+                        if (col + e < d_out)
+                            acc[e] += __bfloat162float(dy_raw[(long long)tau * ldy + col + e]);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 4);
+                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 8);
+                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+            }
+            if (rsub == 0) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) red[ew * 32 + cq * 8 + e] = acc[e];
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(BIAS_WARPS * 32) : "memory");
+            if (ew == 0) {
+                const int qcol = slab * 32 + lane;
+                if (qcol < d_out) {
+                    float g = 0.f;
+#pragma unroll
+                    for (int w2 = 0; w2 < BIAS_WARPS; ++w2) g += red[w2 * 32 + lane];
+                    bias_m[qcol] = fmaf(a, g, bias_m[qcol]);
+                    bias_v[qcol] = fmaf(b * g, g, bias_v[qcol]);
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(BIAS_WARPS * 32) : "memory");
+        }
     } else {
         // ---------------- epilogue: m = fma(a, G, m), v = fma(b*G, G, v) ----------------
         const int q = warp & 3;            // TMEM lane quarter this warp may read
         const int part = (warp - 2) >> 2;  // which part of the tile's columns it handles
-        const int col_split = ((int)blockDim.x / 32 - 2) / 4;  // 1 or 2 warps per lane quarter
+        const int col_split = epi_warps / 4;  // 1 or 2 warps per lane quarter
         const uint32_t sm_g = base + G::SMEM_EPI_OFF + (uint32_t)(warp - 2) * EPI_BUF_BYTES;
         // staging buffer: 32 rows of 128 bytes; 16-byte chunk j of row r sits at (j ^ (r & 7)),
         // which makes both the row-per-thread writes and the row-segment reads conflict-free
@@ -797,11 +897,12 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     }
     const int groups = items < max_groups ? items : max_groups;
     // 8 epilogue warps when no CTA group gets a second tile (exposed epilogue), else 4
-    const int threads = 32 * (2 + (items <= max_groups ? MAX_EPI_WARPS : 4));
+    const int threads = 32 * (2 + (items <= max_groups ? MAX_EPI_WARPS : 4) + (p.bias_m ? BIAS_WARPS : 0));
     if (g_variant == 1) {
         wgrad_fold_kernel<1><<<groups, threads, Geo<1>::SMEM_BYTES, p.stream>>>(
             map_x, map_dy, map_x3, map_dy3, map_dy3h, 0, p.m, p.v, (long long)p.ldmv, p.tokens,
-            p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status);
+            p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status,
+            static_cast<const __nv_bfloat16 *>(p.dY), (long long)p.ldy, p.bias_m, p.bias_v);
         return cudaGetLastError();
     }
     cudaLaunchConfig_t cfg = {};
@@ -819,7 +920,8 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_x3, map_dy3, map_dy3h,
                               grouped, p.m, p.v,
                               (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
-                              p.c.a, p.c.b, p.status);
+                              p.c.a, p.c.b, p.status, static_cast<const __nv_bfloat16 *>(p.dY),
+                              (long long)p.ldy, p.bias_m, p.bias_v);
 }
 
 }  // namespace adama
