@@ -489,7 +489,8 @@ def run_stack(args):
     torch.cuda.set_device(dev)
     pk = peaks()
     if args.workload == "gpt2xl":
-        stack, tokens, n_micro, cfg_id = gpt2xl_stack(wl.CONFIG4_BLOCKS), wl.CONFIG4_TOKENS, wl.CONFIG4_N_MICRO, 4
+        stack, tokens, n_micro, cfg_id = (gpt2xl_stack(wl.CONFIG4_BLOCKS, biases=args.biases), wl.CONFIG4_TOKENS,
+                                          wl.CONFIG4_N_MICRO, 4)
     else:
         stack, tokens, n_micro, cfg_id = llama7b_stack(wl.CONFIG5_BLOCKS), wl.CONFIG5_TOKENS, wl.CONFIG5_N_MICRO, 5
     stack.w.normal_(0, 0.02, generator=torch.Generator(device=dev).manual_seed(wl.seed_for(cfg_id, 99)))
@@ -558,7 +559,8 @@ def run_stack(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate and state",
         "data": "synthetic",
-        "config": {"workload": args.workload, "layers": len(stack.layers), "params": stack.n_params,
+        "config": {"workload": args.workload, "biases": bool(getattr(stack, "biases", False)),
+                   "layers": len(stack.layers), "params": stack.n_params,
                    "tokens_per_micro_batch": tokens, "n_micro": n_micro,
                    "l2": "inputs larger than L2, no flush"},
         "roofline": {"kernel": "wgrad_fold_kernel<2>", "bound": "tensor", "achieved": tf,
@@ -787,6 +789,8 @@ def main():
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--biases", action="store_true",
+                    help="gpt2xl workload: give every linear layer a bias, folded in the fused launch")
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
     ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

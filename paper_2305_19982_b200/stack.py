@@ -5,7 +5,7 @@ layer's [d_in, d_out] matrix back to back; each layer is a view.  One mini-batch
 follows Algorithm 2 of the AdamA paper: for every micro-batch the layers are
 visited from the last to the first (the order in which backward produces their
 gradients), each layer's (X, dY) pair is handed to the fused weight-gradient fold
-and dropped at once, and after the last micro-batch every parameter is updated.
+(which also folds the layer's bias gradient when the stack has biases) and dropped at once, and after the last micro-batch every parameter is updated.
 This module only sequences library calls and owns memory; all arithmetic is in
 the CUDA kernels.
 """
@@ -27,15 +27,20 @@ class LayerSpec:
 
 
 class LinearStack:
-    def __init__(self, layers: Sequence[LayerSpec], device="cuda"):
+    def __init__(self, layers: Sequence[LayerSpec], device="cuda", biases: bool = False):
         self.layers: List[LayerSpec] = list(layers)
         self.device = torch.device(device)
+        self.biases = biases
         self.offsets: List[int] = []
+        self.bias_offsets: List[int] = []
         total = 0
         for L in self.layers:
             self.offsets.append(total)
             total += L.d_in * L.d_out
             total = (total + 63) // 64 * 64  # keep every layer 256-byte aligned
+            if biases:  # the layer's bias [d_out] follows its matrix
+                self.bias_offsets.append(total)
+                total = (total + L.d_out + 63) // 64 * 64
         self.numel = total
         self.w = torch.zeros(total, dtype=torch.float32, device=self.device)
         self.m = torch.zeros(total, dtype=torch.float32, device=self.device)
@@ -43,7 +48,11 @@ class LinearStack:
 
     @property
     def n_params(self) -> int:
-        return sum(L.d_in * L.d_out for L in self.layers)
+        return sum(L.d_in * L.d_out + (L.d_out if self.biases else 0) for L in self.layers)
+
+    def bias_view(self, buf: torch.Tensor, j: int) -> torch.Tensor:
+        o = self.bias_offsets[j]
+        return buf[o:o + self.layers[j].d_out]
 
     def view(self, buf: torch.Tensor, j: int) -> torch.Tensor:
         L = self.layers[j]
@@ -70,22 +79,28 @@ class LinearStack:
                 spec = self.layers[j]
                 X, dY = inputs(i, j, spec)
                 if materialise == "none":
-                    opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j))
+                    if self.biases:  # bias gradient (column sums of dY) in the same launch
+                        opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j),
+                                              self.bias_view(self.m, j), self.bias_view(self.v, j))
+                    else:
+                        opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j))
                 else:
                     G = torch.empty(spec.d_in, spec.d_out, dtype=torch.float32, device=self.device)
                     torch.mm(X.t(), dY, out_dtype=torch.float32, out=G)
                     opt.fold(G.view(-1), self.view(self.m, j).view(-1), self.view(self.v, j).view(-1))
                     del G
+                    if self.biases:
+                        opt.bias_grad_fold(dY, self.bias_view(self.m, j), self.bias_view(self.v, j))
                 del X, dY
         # one apply over the whole flat buffer (padding between layers holds zeros)
         opt.apply(self.w, self.m, self.v, lr)
 
 
-def gpt2xl_stack(blocks: int, device="cuda") -> LinearStack:
+def gpt2xl_stack(blocks: int, device="cuda", biases: bool = False) -> LinearStack:
     h = 1600
     per_block = [("qkv", h, 3 * h), ("out_proj", h, h), ("fc1", h, 4 * h), ("fc2", 4 * h, h)]
     return LinearStack([LayerSpec(f"b{b}.{n}", di, do) for b in range(blocks)
-                        for (n, di, do) in per_block], device)
+                        for (n, di, do) in per_block], device, biases)
 
 
 def llama7b_stack(blocks: int, device="cuda") -> LinearStack:

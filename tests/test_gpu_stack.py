@@ -18,14 +18,14 @@ pytestmark = pytest.mark.gpu
 TOL_BF16 = 2e-3
 
 
-def test_small_stack_full_parity():
+@pytest.mark.parametrize("biases,materialise", [(False, "none"), (True, "none"), (True, "layer")])
+def test_small_stack_full_parity(biases, materialise):
     layers = [LayerSpec("a", 200, 328), LayerSpec("b", 328, 136), LayerSpec("c", 136, 8)]
     T, N, steps = 192, 2, 2
-    stack = LinearStack(layers)
+    stack = LinearStack(layers, biases=biases)
     stack.w.normal_(0, 0.02, generator=torch.Generator(device="cuda").manual_seed(5))
-    for j in range(len(layers)):        # padding between layers stays zero
-        pass
     orcs = [AdamAOracle(f64(stack.view(stack.w, j))) for j in range(len(layers))]
+    borcs = [AdamAOracle(f64(stack.bias_view(stack.w, j))) for j in range(len(layers))] if biases else []
     opt = adama.AdamA()
     order = []
     for step in range(steps):
@@ -35,11 +35,20 @@ def test_small_stack_full_parity():
             dY = wl.normal((T, spec.d_out), 1e-2, torch.bfloat16, wl.seed_for(4, step, i, j) + 50)
             if i == 0:
                 orcs[j].begin_minibatch(N)
+                if biases:
+                    borcs[j].begin_minibatch(N)
             orcs[j].fold_linear(f64(X), f64(dY))
+            if biases:      # bias gradient = column sums of dY (naive loop in the oracle)
+                borcs[j].fold(oracle.linear_wgrad(np.ones((T, 1)), f64(dY))[0])
             return X.cuda(), dY.cuda()
-        stack.minibatch(opt, N, wl.LR, inputs)
+        stack.minibatch(opt, N, wl.LR, inputs, materialise=materialise)
         opt.sync_status()
         for j in range(len(layers)):
+            if biases:
+                borcs[j].update(wl.LR)
+                assert rel_l2(f64(stack.bias_view(stack.w, j)), borcs[j].theta) <= TOL_BF16
+                assert rel_l2(f64(stack.bias_view(stack.m, j)), wl.BETA1 * borcs[j].m) <= TOL_BF16
+                assert rel_l2(f64(stack.bias_view(stack.v, j)), wl.BETA2 * borcs[j].v) <= TOL_BF16
             orcs[j].update(wl.LR)
             assert rel_l2(f64(stack.view(stack.w, j)), orcs[j].theta) <= TOL_BF16
             assert rel_l2(f64(stack.view(stack.m, j)), wl.BETA1 * orcs[j].m) <= TOL_BF16
