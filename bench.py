@@ -629,8 +629,8 @@ def run_sweep(args):
 
 def run_extensions(args):
     """The kernels beside the headline path at the flat workload's size (335 M elements, inputs far
-    above the L2): SGD-momentum fold / apply, the coefficient statistics, apply with the bf16
-    copy.  Median of 20 launches each, CUDA events, against the same HBM peak."""
+    above the L2): the fold with fp32 gradients, SGD-momentum fold / apply, the coefficient
+    statistics, apply with the bf16 copy.  Median of 20 launches each, CUDA events, against the same HBM peak."""
     import paper_2305_19982_b200 as adama
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
@@ -647,7 +647,9 @@ def run_extensions(args):
     wb = torch.empty(n, dtype=torch.bfloat16, device=dev)
     stats = torch.zeros(4, dtype=torch.float64, device=dev)
     rows = {}
+    g32 = wl.normal((n,), wl.CONFIG2.grad_std, torch.float32, 6, device=dev)
     for name, call, bpp in (
+            ("fold_f32_gradients", lambda: opt.fold(g32, m, v), 20),
             ("sgdm_fold_bf16", lambda: opt.sgdm_fold(g, m), 2 + 8),
             ("sgdm_apply", lambda: opt.sgdm_apply(w, m, 1e-3, 0.9), 16),
             ("coefficient_stats", lambda: opt.coefficient_stats(m, m0, v, va, stats), 20),
