@@ -216,6 +216,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
             : "memory");
     }
 }
+// Programmatic dependent launch.  grid_dependency_wait: returns once the kernel launched before
+// this one in the stream has completed and its writes are visible (at once if this launch was
+// not made programmatic).  grid_launch_dependents: the next kernel in the stream, if it was
+// launched programmatic, may start its CTAs as soon as this grid's CTAs have all got here or
+// exited and an SM is free.
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -441,10 +452,16 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     if constexpr (CTAS == 2) cluster_sync_all();  // the partner's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
+    // Everything above touched only this CTA's shared and tensor memory, so it may run while
+    // the previous kernel of the stream is still finishing; every role that reads or writes
+    // global memory waits for that kernel first.  The next kernel may in turn set itself up
+    // on SMs that this grid's CTAs leave early (the last round rarely fills all of them).
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ---------------- TMA producer (one thread of every CTA) ----------------
         if (lane == 0) {
+            grid_dependency_wait();  // X and dY may come from the kernel just before this one
             int stage = 0;
             uint32_t phase = 0;
             uint32_t armed = 0;        // bit s: stage s has been armed at least once
@@ -596,6 +613,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         // combined across the 8 row lanes by shuffles and across the two warps through shared
         // memory, in fixed order.  These warps wait on no mbarrier, so the named barrier
         // between them cannot be left waiting by a role that gave up.
+        grid_dependency_wait();
         const int ew = warp - (2 + epi_warps);
         const int slabs = (d_out + 31) / 32;
         float *red = reinterpret_cast<float *>(smem + G::SMEM_BIAS_OFF);  // [BIAS_WARPS][32]
@@ -679,6 +697,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         const int c4 = lane & 7;        // which float4 of the 32-column chunk
         bool ok = true;
         int it = 0;
+        grid_dependency_wait();  // m and v may still be written by the previous call
         for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
@@ -787,6 +806,7 @@ EncodeTiledFn g_encode = nullptr;
 bool g_attr_set = false;
 int g_variant = 0;  // 0 = not chosen yet, 1 = one-CTA tiles, 2 = CTA pairs
 bool g_no_grouped = false;
+bool g_no_pdl = false;
 
 // 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
 bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void *ptr,
@@ -842,6 +862,9 @@ cudaError_t wgrad_fold_setup(const char **msg) {
         g_variant = (env && env[0] == '1') ? 1 : 2;
         const char *ng = getenv("ADAMA_WGRAD_NO_GROUPED");
         g_no_grouped = ng && ng[0] == '1';
+        // ADAMA_WGRAD_NO_PDL=1 launches without programmatic stream serialization (comparisons)
+        const char *np = getenv("ADAMA_WGRAD_NO_PDL");
+        g_no_pdl = np && np[0] == '1';
     }
     return cudaSuccess;
 }
@@ -910,13 +933,16 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = Geo<2>::SMEM_BYTES;
     cfg.stream = p.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // programmatic launch: this kernel's set-up may overlap the tail of the kernel before it
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = g_no_pdl ? 1 : 2;
     return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_x3, map_dy3, map_dy3h,
                               grouped, p.m, p.v,
                               (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
