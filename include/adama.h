@@ -72,6 +72,10 @@ typedef enum adama_dtype { ADAMA_F32 = 0, ADAMA_BF16 = 1 } adama_dtype;
 
 /* flags for adama_config.flags */
 #define ADAMA_GRADS_PRESCALED 1u /* gradients already carry the 1/N of Algorithm 2 */
+/* adama_apply_to_host copies the weights back on a stream of the context's own instead of on
+ * `cuda_stream`, so that the copy (device to host) can run while later calls already stream the
+ * next gradients in (host to device); see adama_apply_to_host for what the caller gives up. */
+#define ADAMA_ASYNC_COPYBACK 2u
 
 typedef struct adama_config {
     double beta1;   /* in [0,1)                                    */
@@ -278,7 +282,13 @@ ADAMA_API adama_status adama_linear_wgrad_fold_host(adama_ctx *ctx, const void *
                                                     void *cuda_stream);
 
 /* adama_apply followed by a device-to-host copy of the updated weights into
- * w_host (n fp32, pinned memory for full speed), queued on `cuda_stream`. */
+ * w_host (n fp32, pinned memory for full speed), queued on `cuda_stream`.
+ * With ADAMA_ASYNC_COPYBACK the copy is queued on the context's copy-back stream instead,
+ * after the update: `cuda_stream` does not wait for it, so the host-to-device copies of
+ * later *_host calls overlap it (the two directions of the link run at once).  The caller
+ * then must not write w, nor read w_host, until one of these has happened on this context:
+ * the next adama_apply* / adama_sgdm_apply call (it makes its stream wait for the copy),
+ * or adama_sync_status (it returns after the copy has finished). */
 ADAMA_API adama_status adama_apply_to_host(adama_ctx *ctx, float *w, float *m, float *v, size_t n,
                                            double lr, float *w_host, void *cuda_stream);
 

@@ -15,6 +15,9 @@ struct adama_ctx {
     int sm_count;
     unsigned *status_dev;      // 256-byte device status block
     cudaStream_t copy_stream;  // host-buffer variants: H2D copies overlap the folds
+    cudaStream_t d2h_stream;   // ADAMA_ASYNC_COPYBACK: weights go back to the host here
+    cudaEvent_t ev_applied, ev_d2h_done;
+    bool d2h_pending;          // a copy-back that no stream has been made to wait for yet
     cudaEvent_t ev_copied[2], ev_folded[2], ev_entry;
     int64_t launches;
     double weight_decay;  // decoupled (AdamW) decay; 0 = the paper's plain update
@@ -86,10 +89,18 @@ struct DeviceGuard {
 
 size_t dtype_size(adama_dtype d) { return d == ADAMA_F32 ? 4 : 2; }
 
+// ADAMA_ASYNC_COPYBACK: before `stream` may overwrite weights, it waits for the copy-back that
+// is still reading them.
+cudaError_t join_copyback(adama_ctx *ctx, cudaStream_t stream) {
+    if (!ctx->d2h_pending) return cudaSuccess;
+    ctx->d2h_pending = false;
+    return cudaStreamWaitEvent(stream, ctx->ev_d2h_done, 0);
+}
+
 bool config_ok(const adama_config *cfg) {
     return cfg && cfg->beta1 >= 0.0 && cfg->beta1 < 1.0 && cfg->beta2 >= 0.0 && cfg->beta2 < 1.0 &&
            cfg->eps >= 0.0 && isfinite(cfg->eps) && cfg->device >= 0 &&
-           (cfg->flags & ~ADAMA_GRADS_PRESCALED) == 0;
+           (cfg->flags & ~(ADAMA_GRADS_PRESCALED | ADAMA_ASYNC_COPYBACK)) == 0;
 }
 
 adama_status check_fold_args(adama_ctx *ctx, const void *grad, adama_dtype gdt, float *m, float *v,
@@ -173,6 +184,11 @@ adama_status adama_init(adama_ctx **out, const adama_config *cfg) {
             e = cudaEventCreateWithFlags(&ctx->ev_folded[i], cudaEventDisableTiming);
     }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
+    if (e == cudaSuccess && (cfg->flags & ADAMA_ASYNC_COPYBACK)) {
+        e = cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_applied, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_d2h_done, cudaEventDisableTiming);
+    }
     if (e == cudaSuccess) e = adama::wgrad_fold_setup(&msg);
     if (e != cudaSuccess) {
         adama_destroy(ctx);
@@ -187,6 +203,12 @@ adama_status adama_destroy(adama_ctx *ctx) {
     DeviceGuard guard(ctx->cfg.device);
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->d2h_stream) {
+        cudaStreamSynchronize(ctx->d2h_stream);  // a copy-back may still be writing host memory
+        cudaStreamDestroy(ctx->d2h_stream);
+    }
+    if (ctx->ev_applied) cudaEventDestroy(ctx->ev_applied);
+    if (ctx->ev_d2h_done) cudaEventDestroy(ctx->ev_d2h_done);
     for (int i = 0; i < 2; ++i) {
         if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
         if (ctx->ev_folded[i]) cudaEventDestroy(ctx->ev_folded[i]);
@@ -280,8 +302,10 @@ static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, siz
     adama::ApplyConstants c = adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2,
                                                           ctx->cfg.eps, ctx->t, lr, world, sharded,
                                                           ctx->weight_decay);
-    cudaError_t e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
-                                        static_cast<cudaStream_t>(cuda_stream), w_bf16_out);
+    cudaError_t e = join_copyback(ctx, static_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaSuccess)
+        e = adama::launch_apply(w, m, v, n, c, ctx->sm_count,
+                                static_cast<cudaStream_t>(cuda_stream), w_bf16_out);
     if (e != cudaSuccess) return cuda_fail(ctx, "apply launch", e);
     ctx->launches += 1;
     return ADAMA_OK;
@@ -336,9 +360,10 @@ adama_status adama_apply_sharded_peers(adama_ctx *ctx, float *const *w_peers, fl
     const adama::ApplyConstants c =
         adama::make_apply_constants(ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->t, lr,
                                     world_size, true, ctx->weight_decay);
-    cudaError_t e = adama::launch_apply_sharded_peers(w_peers, m_peers, v_peers, world_size, rank, n,
-                                                      c, ctx->sm_count,
-                                                      static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = join_copyback(ctx, static_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaSuccess)
+        e = adama::launch_apply_sharded_peers(w_peers, m_peers, v_peers, world_size, rank, n, c,
+                                              ctx->sm_count, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "apply_sharded_peers launch", e);
     ctx->launches += 1;
     return ADAMA_OK;
@@ -425,7 +450,7 @@ adama_status adama_apply_multi(adama_ctx *ctx, float *const *w, float *const *m,
     float *w_[adama::kMultiMax], *m_[adama::kMultiMax], *v_[adama::kMultiMax];
     size_t n_[adama::kMultiMax];
     int k = 0;
-    cudaError_t e = cudaSuccess;
+    cudaError_t e = join_copyback(ctx, stream);
     for (int i = 0; i <= count && e == cudaSuccess; ++i) {
         const bool flush = (i == count) || k == adama::kMultiMax;
         if (flush && k > 0) {
@@ -533,8 +558,18 @@ adama_status adama_apply_to_host(adama_ctx *ctx, float *w, float *m, float *v, s
     adama_status st = adama_apply(ctx, w, m, v, n, lr, cuda_stream);
     if (st != ADAMA_OK || n == 0) return st;
     DeviceGuard guard(ctx->cfg.device);
-    cudaError_t e = cudaMemcpyAsync(w_host, w, n * sizeof(float), cudaMemcpyDeviceToHost,
-                                    static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e;
+    if (ctx->cfg.flags & ADAMA_ASYNC_COPYBACK) {
+        e = cudaEventRecord(ctx->ev_applied, stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->d2h_stream, ctx->ev_applied, 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(w_host, w, n * sizeof(float), cudaMemcpyDeviceToHost, ctx->d2h_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_d2h_done, ctx->d2h_stream);
+        if (e == cudaSuccess) ctx->d2h_pending = true;
+    } else {
+        e = cudaMemcpyAsync(w_host, w, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, "apply_to_host copy", e);
     return ADAMA_OK;
 }
@@ -576,8 +611,10 @@ adama_status adama_sgdm_apply(adama_ctx *ctx, float *w, float *buf, size_t n, do
     DeviceGuard guard(ctx->cfg.device);
     float mu_hi, mu_lo;
     adama::split_hi_lo(momentum, &mu_hi, &mu_lo);
-    cudaError_t e = adama::launch_sgdm_apply(w, buf, n, (float)lr, mu_hi, mu_lo, ctx->sm_count,
-                                             static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = join_copyback(ctx, static_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaSuccess)
+        e = adama::launch_sgdm_apply(w, buf, n, (float)lr, mu_hi, mu_lo, ctx->sm_count,
+                                     static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "sgdm_apply launch", e);
     ctx->launches += 1;
     return ADAMA_OK;
@@ -636,8 +673,9 @@ adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream) {
     DeviceGuard guard(ctx->cfg.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     unsigned host[4] = {0, 0, 0, 0};
-    cudaError_t e =
-        cudaMemcpyAsync(host, ctx->status_dev, sizeof(host), cudaMemcpyDeviceToHost, stream);
+    cudaError_t e = join_copyback(ctx, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(host, ctx->status_dev, sizeof(host), cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(ctx, "sync_status", e);
     if (host[0] != adama::kDevOk) {

@@ -3,6 +3,7 @@ the host; nothing here launches a faulty kernel)."""
 import pytest
 import torch
 
+import adama_workloads as wl
 import paper_2305_19982_b200 as adama
 from paper_2305_19982_b200 import Status
 
@@ -128,3 +129,36 @@ def test_checkpoint_resume_is_bit_identical():
     a = run(4)
     b = run(4, resume_after=2)
     assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
+def test_async_copyback_gives_the_same_weights_and_is_ordered_before_the_next_update():
+    """ADAMA_ASYNC_COPYBACK: the device-to-host copy of apply_to_host runs on the context's own
+    stream.  Three mini-batches without any host synchronisation in between: every copy-back
+    must hold the weights of ITS step (the next update has to wait for the copy that is still
+    reading w), and the final state equals the stream-ordered form bit for bit."""
+    n = 8_000_003            # 32 MB: long enough copies for an ordering mistake to show
+    g = [wl.normal((n,), 1e-3, torch.bfloat16, 70 + i).cuda() for i in range(2)]
+    res = {}
+    for mode in (False, True):
+        opt = adama.AdamA(async_copyback=mode)
+        w = wl.normal((n,), 0.02, torch.float32, 71).cuda()
+        m, v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+        hosts = [torch.zeros(n, dtype=torch.float32).pin_memory() for _ in range(3)]
+        snaps = []
+        for step in range(3):
+            opt.begin_minibatch(2)
+            for i in range(2):
+                opt.fold(g[i], m, v)
+            opt.apply_to_host(w, m, v, wl.LR, hosts[step])
+            if not mode:
+                snaps.append(w.clone())     # stream-ordered: what w holds after this step
+        opt.sync_status()
+        torch.cuda.synchronize()
+        res[mode] = (w.cpu(), [h.clone() for h in hosts], [s.cpu() for s in snaps])
+        opt.close()
+    w_sync, hosts_sync, snaps = res[False]
+    w_async, hosts_async, _ = res[True]
+    assert torch.equal(w_sync, w_async)
+    for step in range(3):
+        assert torch.equal(hosts_sync[step], snaps[step])
+        assert torch.equal(hosts_async[step], snaps[step])
