@@ -2,7 +2,7 @@
 """Benchmark of the AdamA hot path on B200: fold / apply GB/s and fused wgrad+fold TFLOP/s.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors|extensions|oracle_timing]
+                    [--workload headline|gpt2xl|llama7b|sweep|small_tensors|extensions|oracle_timing|wgrad_shapes]
 
 One step of the headline workload = one pass of the whole path:
   phase A  (flat 335M-parameter buffer, bf16 gradients, N=8):
@@ -735,6 +735,100 @@ def run_oracle_timing(args):
                       "cpu": cpu, "rows": rows}), flush=True)
 
 
+def run_wgrad_shapes(args):
+    """The fused weight-gradient call on every distinct layer shape of the workloads (4096 tokens),
+    alone, with the bias gradient folded in the same launch, and followed by the separate bias
+    kernel; timed back to back and one call at a time with the L2 flushed."""
+    import paper_2305_19982_b200 as adama
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pk = peaks()
+    T = wl.CONFIG3.tokens
+    shapes = [(wl.CONFIG3.d_in, wl.CONFIG3.d_out)]
+    for _, di, do in list(wl.llama7b_block_linears()) + list(wl.gpt2xl_block_linears()):
+        if (di, do) not in shapes:
+            shapes.append((di, do))
+    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
+    opt.begin_minibatch(4)
+
+    def timed(call, reps=20):
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e3
+
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    def timed_cold(call, reps=10):
+        # one call at a time with the L2 overwritten before it: what a layer costs inside a model
+        # whose states are far larger than the L2
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        ts.sort()
+        return ts[len(ts) // 2]
+
+    rows = []
+    for d_in, d_out in shapes:
+        X = wl.normal((T, d_in), 1.0, torch.bfloat16, 1, device=dev)
+        dY = wl.normal((T, d_out), 1e-2, torch.bfloat16, 2, device=dev)
+        m = torch.zeros(d_in, d_out, device=dev)
+        v = torch.zeros(d_in, d_out, device=dev)
+        mb = torch.zeros(d_out, device=dev)
+        vb = torch.zeros(d_out, device=dev)
+
+        def both():
+            opt.linear_wgrad_fold(X, dY, m, v)
+            opt.bias_grad_fold(dY, mb, vb)
+
+        def rested(fn, call):
+            # a pause before every measurement: under the power cap the SM clock sags after a few
+            # milliseconds of dense tensor work and would carry over into the next shape
+            torch.cuda.synchronize()
+            time.sleep(0.5)
+            return fn(call)
+
+        us = rested(timed, lambda: opt.linear_wgrad_fold(X, dY, m, v))
+        us_fused = rested(timed, lambda: opt.linear_wgrad_fold(X, dY, m, v, mb, vb))
+        us_sep = rested(timed, both)
+        cold = rested(timed_cold, lambda: opt.linear_wgrad_fold(X, dY, m, v))
+        cold_fused = rested(timed_cold, lambda: opt.linear_wgrad_fold(X, dY, m, v, mb, vb))
+        cold_sep = rested(timed_cold, both)
+        tf = 2.0 * T * d_in * d_out / us / 1e6
+        tf_cold = 2.0 * T * d_in * d_out / cold / 1e6
+        rows.append({"d_in": d_in, "d_out": d_out, "tokens": T,
+                     "back_to_back": {"us": us, "TFLOPps": tf,
+                                      "frac_of_burst_peak": tf / pk["bf16_tflops"],
+                                      "us_with_fused_bias": us_fused,
+                                      "us_with_separate_bias_kernel": us_sep},
+                     "l2_flushed": {"us": cold, "TFLOPps": tf_cold,
+                                    "frac_of_burst_peak": tf_cold / pk["bf16_tflops"],
+                                    "us_with_fused_bias": cold_fused,
+                                    "us_with_separate_bias_kernel": cold_sep}})
+        del X, dY, m, v
+    opt.sync_status()
+    print(json.dumps({"metric": "adama_wgrad_fold_per_shape", "unit": "us", "peak_tflops": pk["bf16_tflops"],
+                      "peak_source": pk["source"],
+                      "timing": "back_to_back: 20 calls between two CUDA events (buffers may stay in "
+                                "the L2); l2_flushed: median of 10 single calls, 512 MB written before each",
+                      "rows": rows}), flush=True)
+    opt.close()
+
+
 def run_small_tensors(args):
     """The non-matrix parameters of a GPT-2-XL-shaped model (per block: two norms, four biases;
     432 tensors, 1.0 M elements): one mini-batch of N=8 folds + apply with the multi-tensor
@@ -798,7 +892,7 @@ def main():
     ap.add_argument("--biases", action="store_true",
                     help="gpt2xl workload: give every linear layer a bias, folded in the fused launch")
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
-    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing"])
+    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing", "wgrad_shapes"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -811,6 +905,8 @@ def main():
         run_extensions(args)
     elif args.workload == "oracle_timing":
         run_oracle_timing(args)
+    elif args.workload == "wgrad_shapes":
+        run_wgrad_shapes(args)
     elif args.workload == "small_tensors":
         args.steps = min(args.steps, 10)
         run_small_tensors(args)
