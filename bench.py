@@ -820,8 +820,26 @@ def run_wgrad_shapes(args):
                                     "us_with_fused_bias": cold_fused,
                                     "us_with_separate_bias_kernel": cold_sep}})
         del X, dY, m, v
+    # token sweep on the 4096 x 4096 layer: below ~2000 tokens the call is bound by the 16 B/param
+    # of m, v traffic, above by the tensor cores
+    sweep = []
+    d_in, d_out = wl.CONFIG3.d_in, wl.CONFIG3.d_out
+    m = torch.zeros(d_in, d_out, device=dev)
+    v = torch.zeros(d_in, d_out, device=dev)
+    for tokens in (256, 512, 1024, 2048, 4096, 8192):
+        X = wl.normal((tokens, d_in), 1.0, torch.bfloat16, 3, device=dev)
+        dY = wl.normal((tokens, d_out), 1e-2, torch.bfloat16, 4, device=dev)
+        torch.cuda.synchronize()
+        time.sleep(0.5)
+        us = timed_cold(lambda: opt.linear_wgrad_fold(X, dY, m, v))
+        byts = 16 * d_in * d_out + 2 * tokens * (d_in + d_out)
+        sweep.append({"tokens": tokens, "us": us, "TFLOPps": 2.0 * tokens * d_in * d_out / us / 1e6,
+                      "hbm_GBps": byts / us / 1e3,
+                      "hbm_floor_us": byts / pk["hbm_gbs"] / 1e3,
+                      "tensor_floor_us": 2.0 * tokens * d_in * d_out / pk["bf16_tflops"] / 1e6})
+        del X, dY
     opt.sync_status()
-    print(json.dumps({"metric": "adama_wgrad_fold_per_shape", "unit": "us", "peak_tflops": pk["bf16_tflops"],
+    print(json.dumps({"metric": "adama_wgrad_fold_per_shape", "token_sweep_4096x4096_l2_flushed": sweep, "unit": "us", "peak_tflops": pk["bf16_tflops"],
                       "peak_source": pk["source"],
                       "timing": "back_to_back: 20 calls between two CUDA events (buffers may stay in "
                                 "the L2); l2_flushed: median of 10 single calls, 512 MB written before each",

@@ -806,6 +806,7 @@ EncodeTiledFn g_encode = nullptr;
 bool g_attr_set = false;
 int g_variant = 0;  // 0 = not chosen yet, 1 = one-CTA tiles, 2 = CTA pairs
 bool g_no_grouped = false;
+int g_force_epi_warps = 0;  // ADAMA_WGRAD_EPI_WARPS=4|8 overrides the per-launch choice (comparisons)
 bool g_no_pdl = false;
 
 // 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
@@ -862,6 +863,8 @@ cudaError_t wgrad_fold_setup(const char **msg) {
         g_variant = (env && env[0] == '1') ? 1 : 2;
         const char *ng = getenv("ADAMA_WGRAD_NO_GROUPED");
         g_no_grouped = ng && ng[0] == '1';
+        const char *ew = getenv("ADAMA_WGRAD_EPI_WARPS");
+        g_force_epi_warps = ew && (ew[0] == '4' || ew[0] == '8') ? ew[0] - '0' : 0;
         // ADAMA_WGRAD_NO_PDL=1 launches without programmatic stream serialization (comparisons)
         const char *np = getenv("ADAMA_WGRAD_NO_PDL");
         g_no_pdl = np && np[0] == '1';
@@ -919,8 +922,12 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
         items = tiles + rest;
     }
     const int groups = items < max_groups ? items : max_groups;
-    // 8 epilogue warps when no CTA group gets a second tile (exposed epilogue), else 4
-    const int threads = 32 * (2 + (items <= max_groups ? MAX_EPI_WARPS : 4) + (p.bias_m ? BIAS_WARPS : 0));
+    // 8 epilogue warps when no CTA group gets a second tile (exposed epilogue) or when the
+    // contraction is short (up to 2048 tokens the m, v traffic of the epilogue, not the tensor
+    // cores, bounds the call: 4096x4096 with 1024 tokens 78.9 vs 82.9 us), else 4
+    const bool wide = g_force_epi_warps ? g_force_epi_warps == 8
+                                        : (items <= max_groups || p.tokens <= 2048);
+    const int threads = 32 * (2 + (wide ? MAX_EPI_WARPS : 4) + (p.bias_m ? BIAS_WARPS : 0));
     if (g_variant == 1) {
         wgrad_fold_kernel<1><<<groups, threads, Geo<1>::SMEM_BYTES, p.stream>>>(
             map_x, map_dy, map_x3, map_dy3, map_dy3h, 0, p.m, p.v, (long long)p.ldmv, p.tokens,
