@@ -75,7 +75,7 @@ constexpr int MAX_THREADS = 32 * (2 + MAX_EPI_WARPS + 2);  // + the two optional
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
 constexpr int MAX_STAGES = 12;
-constexpr int SMEM_BAR_BYTES = 256;
+constexpr int SMEM_BAR_BYTES = 512;
 #ifndef ADAMA_WGRAD_BIAS_UNROLL
 #define ADAMA_WGRAD_BIAS_UNROLL 8
 #endif
@@ -83,8 +83,17 @@ constexpr int BIAS_UNROLL = ADAMA_WGRAD_BIAS_UNROLL;  // 16-byte loads in flight
 constexpr int BIAS_WARPS = 2;
 constexpr int SMEM_BIAS_BYTES = BIAS_WARPS * 32 * 4;
 
+// Staged epilogue (calls of few tokens, where the m, v traffic bounds the call): the accumulator
+// tile is first copied into shared memory (128 rows x 256 fp32 = 128 KB per CTA, which a
+// 3-stage ring leaves room for), and separate streaming warps fold it into m and v.
+constexpr int STAGED_RING = 3;
+constexpr int STAGED_DRAIN_WARPS = 4;   // tensor memory -> shared memory, one per lane quarter
+constexpr int STAGED_STREAM_WARPS = 8;  // shared memory -> m, v (16 rows of the tile each)
+constexpr int G_TILE_BYTES = 128 * BN * 4;
+constexpr int STAGED_THREADS = 32 * (2 + STAGED_DRAIN_WARPS + STAGED_STREAM_WARPS + BIAS_WARPS);
+
 // Per-variant geometry: CTAS = CTAs cooperating on one tile (1 or 2).
-template <int CTAS>
+template <int CTAS, bool STAGED = false>
 struct Geo {
     static constexpr int ROWS_PER_CTA = 128;                 // TMEM lanes
     static constexpr int TILE_M = ROWS_PER_CTA * CTAS;       // UMMA M
@@ -94,9 +103,10 @@ struct Geo {
     static constexpr int A_STAGE_BYTES = A_BOXES * BOX_BYTES;
     static constexpr int B_STAGE_BYTES = B_BOXES * BOX_BYTES;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KB or 32 KB
-    static constexpr int STAGES = CTAS == 1 ? 4 * 64 / BK : ADAMA_WGRAD_STAGES;
+    static constexpr int STAGES =
+        STAGED ? STAGED_RING : (CTAS == 1 ? 4 * 64 / BK : ADAMA_WGRAD_STAGES);
     static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
-    static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + EPI_BYTES;
+    static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + (STAGED ? G_TILE_BYTES : EPI_BYTES);
     static constexpr int SMEM_BIAS_OFF = SMEM_BAR_OFF + SMEM_BAR_BYTES;
     static constexpr int SMEM_BYTES = SMEM_BIAS_OFF + SMEM_BIAS_BYTES + 1024;  // + alignment slack
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -367,6 +377,8 @@ struct Barriers {
     uint64_t acc_full[ACC_STAGES];
     uint64_t acc_empty[ACC_STAGES];
     uint64_t drain;
+    uint64_t g_full[2];   // staged epilogue: a 128-column half of the tile in shared memory is complete
+    uint64_t g_empty[2];  // staged epilogue: the streaming warps are done with that half
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -401,8 +413,8 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
     return {(full % tiles_m) * Geo<CTAS>::TILE_M, (full / tiles_m) * BN + half * (BN / 2), width};
 }
 
-template <int CTAS>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
+template <int CTAS, bool STAGED>
+__global__ void __launch_bounds__(STAGED ? STAGED_THREADS : MAX_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   const __grid_constant__ CUtensorMap map_dy,
                   const __grid_constant__ CUtensorMap map_x3,
@@ -413,7 +425,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   int split_from, int num_items, float a, float b, unsigned *status,
                   const __nv_bfloat16 *__restrict__ dy_raw, long long ldy,
                   float *__restrict__ bias_m, float *__restrict__ bias_v) {
-    using G = Geo<CTAS>;
+    using G = Geo<CTAS, STAGED>;
     constexpr int STAGES = G::STAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -430,7 +442,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
     const int num_kb = (tokens + BK - 1) / BK;
     // warps 2 .. 2+epi_warps-1: epilogue; with bias moments, BIAS_WARPS more after them
-    const int epi_warps = (int)blockDim.x / 32 - 2 - (bias_m != nullptr ? BIAS_WARPS : 0);
+    // (staged: 4 drain warps take the epilogue's place, 8 streaming warps follow them)
+    const int epi_warps = STAGED ? STAGED_DRAIN_WARPS
+                                 : (int)blockDim.x / 32 - 2 - (bias_m != nullptr ? BIAS_WARPS : 0);
+    const int first_bias_warp = 2 + epi_warps + (STAGED ? STAGED_STREAM_WARPS : 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -442,6 +457,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             mbar_init(smem_u32(&bars->acc_empty[s]), epi_warps * CTAS);
         }
         mbar_init(smem_u32(&bars->drain), 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(smem_u32(&bars->g_full[h]), STAGED_DRAIN_WARPS);
+            mbar_init(smem_u32(&bars->g_empty[h]), STAGED_STREAM_WARPS);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -602,7 +621,86 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             }
         }
         __syncwarp();
-    } else if (warp >= 2 + epi_warps) {
+    } else if (STAGED && warp >= 2 + STAGED_DRAIN_WARPS && warp < 2 + STAGED_DRAIN_WARPS + STAGED_STREAM_WARPS) {
+        // ---------------- staged epilogue, streaming side: shared-memory tile -> m, v ----------------
+        // A warp owns 16 rows of the CTA's 128; the tile comes in two 128-column halves, so that
+        // one half is folded while the drain warps copy the other.  A warp instruction covers 512
+        // contiguous bytes of one row; eight rows of m and of v are in flight per thread.
+        const int sw_id = warp - (2 + STAGED_DRAIN_WARPS);
+        const uint32_t gbuf = base + G::SMEM_EPI_OFF;
+        bool ok = true;
+        uint32_t use_bits = 0;  // bit h: parity of how often half h of the tile buffer has been used
+        grid_dependency_wait();     // m and v may still be written by the previous call
+        for (int tile = group; tile < num_items && ok; tile += num_groups) {
+            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+            const int row_base = wi.m0 + (int)rank * G::ROWS_PER_CTA;
+            for (int h = 0; h < wi.width / 128; ++h) {
+                if (!ok) continue;
+                ok = mbar_wait(smem_u32(&bars->g_full[h]), (use_bits >> h) & 1u, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) {
+                    if (lane == 0) record_timeout(status, bars, 7, (unsigned)tile);
+                    continue;
+                }
+                use_bits ^= 1u << h;
+                const int gcol = wi.n0 + h * 128 + lane * 4;
+                const bool col_vec = gcol + 4 <= d_out;  // whole group of four columns inside
+                for (int rb = 0; rb < 16; rb += 8) {
+                    const int lrow0 = sw_id * 16 + rb;
+                    int rows_ok = d_in - (row_base + lrow0);  // rows of this batch inside the matrix
+                    rows_ok = rows_ok < 0 ? 0 : (rows_ok > 8 ? 8 : rows_ok);
+                    float *pm = m_out + (long long)(row_base + lrow0) * ldmv + gcol;
+                    float *pv = v_out + (long long)(row_base + lrow0) * ldmv + gcol;
+                    float4 mm[8], vv[8];
+                    if (col_vec) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i < rows_ok) {
+                                mm[i] = ld_global_v4_stream(pm + (long long)i * ldmv);
+                                vv[i] = ld_global_v4_stream(pv + (long long)i * ldmv);
+                            }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i < rows_ok) {
+                                const int lrow = lrow0 + i;
+                                const float4 g =
+                                    ld_shared_v4(gbuf + (uint32_t)lrow * 1024u +
+                                                 (uint32_t)(((h * 32 + lane) ^ (lrow & 7)) << 4));
+                                float4 &x = mm[i], &y = vv[i];
+                                x.x = fmaf(a, g.x, x.x);
+                                x.y = fmaf(a, g.y, x.y);
+                                x.z = fmaf(a, g.z, x.z);
+                                x.w = fmaf(a, g.w, x.w);
+                                y.x = fmaf(b * g.x, g.x, y.x);
+                                y.y = fmaf(b * g.y, g.y, y.y);
+                                y.z = fmaf(b * g.z, g.z, y.z);
+                                y.w = fmaf(b * g.w, g.w, y.w);
+                                st_global_v4(pm + (long long)i * ldmv, x);
+                                st_global_v4(pv + (long long)i * ldmv, y);
+                            }
+                    } else if (gcol < d_out) {
+                        // last, partial group of four columns: element-wise
+                        for (int i = 0; i < rows_ok; ++i) {
+                            const int lrow = lrow0 + i;
+                            const float4 g =
+                                ld_shared_v4(gbuf + (uint32_t)lrow * 1024u +
+                                             (uint32_t)(((h * 32 + lane) ^ (lrow & 7)) << 4));
+                            const float ge[4] = {g.x, g.y, g.z, g.w};
+                            for (int e = 0; e < 4; ++e)
+                                if (gcol + e < d_out) {
+                                    float *qm = pm + (long long)i * ldmv + e;
+                                    float *qv = pv + (long long)i * ldmv + e;
+                                    *qm = fmaf(a, ge[e], *qm);
+                                    *qv = fmaf(b * ge[e], ge[e], *qv);
+                                }
+                        }
+                    }
+                }
+                __syncwarp();  // every lane has read its part of this half
+                if (lane == 0) mbar_arrive(smem_u32(&bars->g_empty[h]));
+            }
+        }
+    } else if (warp >= first_bias_warp) {
         // ---------------- bias gradient: column sums of dY, folded into the bias moments ----------------
         // Two extra warps (present only when bias moments were passed) work through the layer's
         // bias gradient while the other roles run the tiles, straight from global memory (the
@@ -614,7 +712,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         // memory, in fixed order.  These warps wait on no mbarrier, so the named barrier
         // between them cannot be left waiting by a role that gave up.
         grid_dependency_wait();
-        const int ew = warp - (2 + epi_warps);
+        const int ew = warp - first_bias_warp;
         const int slabs = (d_out + 31) / 32;
         float *red = reinterpret_cast<float *>(smem + G::SMEM_BIAS_OFF);  // [BIAS_WARPS][32]
         const int rsub = lane >> 2;  // row within a group of 8
@@ -683,6 +781,64 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             asm volatile("bar.sync 1, %0;" ::"r"(BIAS_WARPS * 32) : "memory");
         }
     } else {
+        if constexpr (STAGED) {
+            // ---------------- staged epilogue, drain side: accumulator -> shared-memory tile ----------------
+            // Thread = accumulator row; 16-byte chunk j of row r sits at chunk (j ^ (r & 7)), so these
+            // row-per-thread writes and the streaming warps' row-contiguous reads are conflict-free.
+            const int q = warp & 3;
+            const uint32_t gbuf = base + G::SMEM_EPI_OFF;
+            const int lrow = q * EPI_ROWS + lane;
+            bool ok = true;
+            int it = 0;
+            uint32_t use_bits = 0;  // bit h: parity of how often half h of the tile buffer has been filled
+            for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
+                const int as = it & 1;
+                const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+                ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) {
+                    if (lane == 0) record_timeout(status, bars, 4, (unsigned)tile);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t taddr0 =
+                    tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
+                for (int h = 0; h < wi.width / 128; ++h) {
+                    if (!ok) continue;
+                    // the streaming warps must be done with this half's previous contents
+                    ok = mbar_wait(smem_u32(&bars->g_empty[h]), ((use_bits >> h) & 1u) ^ 1u, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) {
+                        if (lane == 0) record_timeout(status, bars, 6, (unsigned)tile);
+                        continue;
+                    }
+                    use_bits ^= 1u << h;
+                    for (int c = h * 4; c < h * 4 + 4; ++c) {
+                        uint32_t r[32];
+                        tc_ld_32x32(taddr0 + (uint32_t)(c * EPI_COLS), r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            st_shared_v4(gbuf + (uint32_t)lrow * 1024u +
+                                             (uint32_t)(((c * 8 + j) ^ (lrow & 7)) << 4),
+                                         __uint_as_float(r[4 * j + 0]), __uint_as_float(r[4 * j + 1]),
+                                         __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->g_full[h]));
+                }
+                if (!ok) break;
+                // the accumulator stage may be overwritten
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    const uint32_t e = smem_u32(&bars->acc_empty[as]);
+                    if constexpr (CTAS == 1) mbar_arrive(e);
+                    else mbar_arrive_cluster(map_to_cta(e, 0));
+                }
+            }
+        } else {
         // ---------------- epilogue: m = fma(a, G, m), v = fma(b*G, G, v) ----------------
         const int q = warp & 3;            // TMEM lane quarter this warp may read
         const int part = (warp - 2) >> 2;  // which part of the tile's columns it handles
@@ -783,6 +939,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 else mbar_arrive_cluster(map_to_cta(e, 0));
             }
         }
+        }  // !STAGED
     }
 
     tc_fence_before();
@@ -808,6 +965,7 @@ int g_variant = 0;  // 0 = not chosen yet, 1 = one-CTA tiles, 2 = CTA pairs
 bool g_no_grouped = false;
 int g_force_epi_warps = 0;  // ADAMA_WGRAD_EPI_WARPS=4|8 overrides the per-launch choice (comparisons)
 bool g_no_pdl = false;
+int g_force_staged = 0;  // ADAMA_WGRAD_STAGED=1|0 forces / forbids the staged epilogue (comparisons)
 
 // 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
 bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void *ptr,
@@ -868,6 +1026,8 @@ cudaError_t wgrad_fold_setup(const char **msg) {
         // ADAMA_WGRAD_NO_PDL=1 launches without programmatic stream serialization (comparisons)
         const char *np = getenv("ADAMA_WGRAD_NO_PDL");
         g_no_pdl = np && np[0] == '1';
+        const char *sg = getenv("ADAMA_WGRAD_STAGED");
+        g_force_staged = sg ? (sg[0] == '1' ? 1 : -1) : 0;
     }
     return cudaSuccess;
 }
@@ -876,11 +1036,15 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cudaError_t e = wgrad_fold_setup(msg);
     if (e != cudaSuccess) return e;
     if (!g_attr_set) {
-        e = cudaFuncSetAttribute(wgrad_fold_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Geo<1>::SMEM_BYTES);
+        e = cudaFuncSetAttribute(wgrad_fold_kernel<1, false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<1>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(wgrad_fold_kernel<2>,
+            e = cudaFuncSetAttribute(wgrad_fold_kernel<2, false>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(wgrad_fold_kernel<2, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Geo<2, true>::SMEM_BYTES);
         if (e != cudaSuccess) {
             *msg = "cudaFuncSetAttribute(wgrad_fold_kernel)";
             return e;
@@ -929,7 +1093,7 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
                                         : (items <= max_groups || p.tokens <= 2048);
     const int threads = 32 * (2 + (wide ? MAX_EPI_WARPS : 4) + (p.bias_m ? BIAS_WARPS : 0));
     if (g_variant == 1) {
-        wgrad_fold_kernel<1><<<groups, threads, Geo<1>::SMEM_BYTES, p.stream>>>(
+        wgrad_fold_kernel<1, false><<<groups, threads, Geo<1>::SMEM_BYTES, p.stream>>>(
             map_x, map_dy, map_x3, map_dy3, map_dy3h, 0, p.m, p.v, (long long)p.ldmv, p.tokens,
             p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status,
             static_cast<const __nv_bfloat16 *>(p.dY), (long long)p.ldy, p.bias_m, p.bias_v);
@@ -938,7 +1102,12 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
-    cfg.dynamicSmemBytes = Geo<2>::SMEM_BYTES;
+    // calls of few tokens: staged epilogue (see STAGED_RING)
+    // (4096x4096, L2 flushed, staged vs not: 256 tokens 65.6 vs 75.8 us, 1024 tokens 71.7 vs 79.9,
+    // 2048 tokens 92.1 vs 82.0 -- there the 3-stage ring starves the main loop)
+    const bool staged = g_force_staged ? g_force_staged > 0 : p.tokens <= 1024;
+    cfg.dynamicSmemBytes = staged ? Geo<2, true>::SMEM_BYTES : Geo<2>::SMEM_BYTES;
+    if (staged) cfg.blockDim = dim3((unsigned)(STAGED_THREADS - (p.bias_m ? 0 : 32 * BIAS_WARPS)), 1, 1);
     cfg.stream = p.stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -950,7 +1119,7 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_no_pdl ? 1 : 2;
-    return cudaLaunchKernelEx(&cfg, wgrad_fold_kernel<2>, map_x, map_dy, map_x3, map_dy3, map_dy3h,
+    return cudaLaunchKernelEx(&cfg, staged ? wgrad_fold_kernel<2, true> : wgrad_fold_kernel<2, false>, map_x, map_dy, map_x3, map_dy3, map_dy3h,
                               grouped, p.m, p.v,
                               (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
                               p.c.a, p.c.b, p.status, static_cast<const __nv_bfloat16 *>(p.dY),

@@ -114,6 +114,15 @@ def test_ragged_shapes(T, d_in, d_out):
     _full_parity(T, d_in, d_out, integer=True, pad=5)
 
 
+@pytest.mark.parametrize("T", [1030, 1100, 2100])
+@pytest.mark.parametrize("d_in,d_out", [(200, 328), (129, 263), (136, 520), (300, 1000)])
+def test_ragged_shapes_beyond_the_short_call_path(T, d_in, d_out):
+    """Calls of up to 1024 tokens take the staged epilogue (accumulator -> shared memory ->
+    streaming fold); these token counts take the direct epilogue instead, on the same ragged
+    shapes and padded buffers.  Integer inputs: exact contraction, fp32 fold tolerance."""
+    _full_parity(T, d_in, d_out, integer=True, pad=5)
+
+
 def test_multi_tile_normal_inputs_two_steps():
     _full_parity(512, 384, 768, n_micro=2, steps=2)
 
