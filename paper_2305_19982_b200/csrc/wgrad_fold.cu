@@ -84,12 +84,18 @@ constexpr int BIAS_WARPS = 2;
 constexpr int SMEM_BIAS_BYTES = BIAS_WARPS * 32 * 4;
 
 // Staged epilogue (calls of few tokens, where the m, v traffic bounds the call): the accumulator
-// tile is first copied into shared memory (128 rows x 256 fp32 = 128 KB per CTA, which a
-// 3-stage ring leaves room for), and separate streaming warps fold it into m and v.
-constexpr int STAGED_RING = 3;
+// tile is first copied into shared memory, part by part (128 rows x PART_COLS fp32, two part
+// buffers, the rest of the shared memory stays with the ring), and separate streaming warps
+// fold the parts into m and v.
+#ifndef ADAMA_WGRAD_PART_COLS
+#define ADAMA_WGRAD_PART_COLS 64
+#endif
+constexpr int PART_COLS = ADAMA_WGRAD_PART_COLS;        // columns of one part of the tile copy
+constexpr int PART_BYTES = 128 * PART_COLS * 4;         // 128 rows: 32 KB (64 columns) or 64 KB (128)
+constexpr int STAGED_RING = (224 * 1024 - 2 * PART_BYTES) / (32 * 1024);  // 5 or 3 stages
 constexpr int STAGED_DRAIN_WARPS = 4;   // tensor memory -> shared memory, one per lane quarter
 constexpr int STAGED_STREAM_WARPS = 8;  // shared memory -> m, v (16 rows of the tile each)
-constexpr int G_TILE_BYTES = 128 * BN * 4;
+constexpr int G_TILE_BYTES = 2 * PART_BYTES;  // two parts: one is filled while the other is folded
 constexpr int STAGED_THREADS = 32 * (2 + STAGED_DRAIN_WARPS + STAGED_STREAM_WARPS + BIAS_WARPS);
 
 // Per-variant geometry: CTAS = CTAs cooperating on one tile (1 or 2).
@@ -377,8 +383,8 @@ struct Barriers {
     uint64_t acc_full[ACC_STAGES];
     uint64_t acc_empty[ACC_STAGES];
     uint64_t drain;
-    uint64_t g_full[2];   // staged epilogue: a 128-column half of the tile in shared memory is complete
-    uint64_t g_empty[2];  // staged epilogue: the streaming warps are done with that half
+    uint64_t g_full[2];   // staged epilogue: part buffer k holds a complete part of the tile
+    uint64_t g_empty[2];  // staged epilogue: the streaming warps are done with part buffer k
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -623,49 +629,53 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         __syncwarp();
     } else if (STAGED && warp >= 2 + STAGED_DRAIN_WARPS && warp < 2 + STAGED_DRAIN_WARPS + STAGED_STREAM_WARPS) {
         // ---------------- staged epilogue, streaming side: shared-memory tile -> m, v ----------------
-        // A warp owns 16 rows of the CTA's 128; the tile comes in two 128-column halves, so that
-        // one half is folded while the drain warps copy the other.  A warp instruction covers 512
-        // contiguous bytes of one row; eight rows of m and of v are in flight per thread.
+        // A warp owns 16 rows of the CTA's 128; the tile comes in parts of PART_COLS columns, so
+        // that one part is folded while the drain warps copy the next.  A warp instruction covers
+        // 32/LPR rows x PART_COLS*4 contiguous bytes; eight such loads of m and of v are in flight
+        // per thread.
         const int sw_id = warp - (2 + STAGED_DRAIN_WARPS);
         const uint32_t gbuf = base + G::SMEM_EPI_OFF;
+        constexpr int LPR = PART_COLS / 4;   // lanes per row: a warp instruction covers 32 / LPR rows
+        constexpr int RPI = 32 / LPR;
+        constexpr int PITCH = PART_COLS * 4;  // bytes per row of a part buffer
+        const int sub = lane / LPR, cl = lane % LPR;
         bool ok = true;
-        uint32_t use_bits = 0;  // bit h: parity of how often half h of the tile buffer has been used
-        grid_dependency_wait();     // m and v may still be written by the previous call
+        uint32_t use_bits = 0;    // bit k: parity of how often part buffer k has been used
+        grid_dependency_wait();   // m and v may still be written by the previous call
         for (int tile = group; tile < num_items && ok; tile += num_groups) {
             const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
             const int row_base = wi.m0 + (int)rank * G::ROWS_PER_CTA;
-            for (int h = 0; h < wi.width / 128; ++h) {
+            for (int part_i = 0; part_i < wi.width / PART_COLS; ++part_i) {
                 if (!ok) continue;
-                ok = mbar_wait(smem_u32(&bars->g_full[h]), (use_bits >> h) & 1u, abort_flag);
+                const int k = part_i & 1;
+                ok = mbar_wait(smem_u32(&bars->g_full[k]), (use_bits >> k) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) {
                     if (lane == 0) record_timeout(status, bars, 7, (unsigned)tile);
                     continue;
                 }
-                use_bits ^= 1u << h;
-                const int gcol = wi.n0 + h * 128 + lane * 4;
+                use_bits ^= 1u << k;
+                const uint32_t pbuf = gbuf + (uint32_t)k * PART_BYTES;
+                const int gcol = wi.n0 + part_i * PART_COLS + cl * 4;
                 const bool col_vec = gcol + 4 <= d_out;  // whole group of four columns inside
-                for (int rb = 0; rb < 16; rb += 8) {
-                    const int lrow0 = sw_id * 16 + rb;
-                    int rows_ok = d_in - (row_base + lrow0);  // rows of this batch inside the matrix
-                    rows_ok = rows_ok < 0 ? 0 : (rows_ok > 8 ? 8 : rows_ok);
+                for (int rb = 0; rb < 16; rb += 8 * RPI) {
+                    const int lrow0 = sw_id * 16 + rb + sub;  // this thread's first row of the batch
                     float *pm = m_out + (long long)(row_base + lrow0) * ldmv + gcol;
                     float *pv = v_out + (long long)(row_base + lrow0) * ldmv + gcol;
                     float4 mm[8], vv[8];
                     if (col_vec) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
-                            if (i < rows_ok) {
-                                mm[i] = ld_global_v4_stream(pm + (long long)i * ldmv);
-                                vv[i] = ld_global_v4_stream(pv + (long long)i * ldmv);
+                            if (row_base + lrow0 + i * RPI < d_in) {
+                                mm[i] = ld_global_v4_stream(pm + (long long)(i * RPI) * ldmv);
+                                vv[i] = ld_global_v4_stream(pv + (long long)(i * RPI) * ldmv);
                             }
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
-                            if (i < rows_ok) {
-                                const int lrow = lrow0 + i;
-                                const float4 g =
-                                    ld_shared_v4(gbuf + (uint32_t)lrow * 1024u +
-                                                 (uint32_t)(((h * 32 + lane) ^ (lrow & 7)) << 4));
+                            if (row_base + lrow0 + i * RPI < d_in) {
+                                const int lrow = lrow0 + i * RPI;
+                                const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
+                                                              (uint32_t)((cl ^ (lrow & 7)) << 4));
                                 float4 &x = mm[i], &y = vv[i];
                                 x.x = fmaf(a, g.x, x.x);
                                 x.y = fmaf(a, g.y, x.y);
@@ -675,29 +685,29 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                                 y.y = fmaf(b * g.y, g.y, y.y);
                                 y.z = fmaf(b * g.z, g.z, y.z);
                                 y.w = fmaf(b * g.w, g.w, y.w);
-                                st_global_v4(pm + (long long)i * ldmv, x);
-                                st_global_v4(pv + (long long)i * ldmv, y);
+                                st_global_v4(pm + (long long)(i * RPI) * ldmv, x);
+                                st_global_v4(pv + (long long)(i * RPI) * ldmv, y);
                             }
                     } else if (gcol < d_out) {
                         // last, partial group of four columns: element-wise
-                        for (int i = 0; i < rows_ok; ++i) {
-                            const int lrow = lrow0 + i;
-                            const float4 g =
-                                ld_shared_v4(gbuf + (uint32_t)lrow * 1024u +
-                                             (uint32_t)(((h * 32 + lane) ^ (lrow & 7)) << 4));
+                        for (int i = 0; i < 8; ++i) {
+                            const int lrow = lrow0 + i * RPI;
+                            if (row_base + lrow >= d_in) break;
+                            const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
+                                                          (uint32_t)((cl ^ (lrow & 7)) << 4));
                             const float ge[4] = {g.x, g.y, g.z, g.w};
                             for (int e = 0; e < 4; ++e)
                                 if (gcol + e < d_out) {
-                                    float *qm = pm + (long long)i * ldmv + e;
-                                    float *qv = pv + (long long)i * ldmv + e;
+                                    float *qm = pm + (long long)(i * RPI) * ldmv + e;
+                                    float *qv = pv + (long long)(i * RPI) * ldmv + e;
                                     *qm = fmaf(a, ge[e], *qm);
                                     *qv = fmaf(b * ge[e], ge[e], *qv);
                                 }
                         }
                     }
                 }
-                __syncwarp();  // every lane has read its part of this half
-                if (lane == 0) mbar_arrive(smem_u32(&bars->g_empty[h]));
+                __syncwarp();  // every lane has read its share of this part
+                if (lane == 0) mbar_arrive(smem_u32(&bars->g_empty[k]));
             }
         }
     } else if (warp >= first_bias_warp) {
@@ -790,7 +800,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             const int lrow = q * EPI_ROWS + lane;
             bool ok = true;
             int it = 0;
-            uint32_t use_bits = 0;  // bit h: parity of how often half h of the tile buffer has been filled
+            uint32_t use_bits = 0;  // bit k: parity of how often part buffer k has been filled
             for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
@@ -804,29 +814,32 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 tc_fence_after();
                 const uint32_t taddr0 =
                     tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
-                for (int h = 0; h < wi.width / 128; ++h) {
+                for (int part_i = 0; part_i < wi.width / PART_COLS; ++part_i) {
                     if (!ok) continue;
-                    // the streaming warps must be done with this half's previous contents
-                    ok = mbar_wait(smem_u32(&bars->g_empty[h]), ((use_bits >> h) & 1u) ^ 1u, abort_flag);
+                    const int k = part_i & 1;
+                    // the streaming warps must be done with this buffer's previous contents
+                    ok = mbar_wait(smem_u32(&bars->g_empty[k]), ((use_bits >> k) & 1u) ^ 1u, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) {
                         if (lane == 0) record_timeout(status, bars, 6, (unsigned)tile);
                         continue;
                     }
-                    use_bits ^= 1u << h;
-                    for (int c = h * 4; c < h * 4 + 4; ++c) {
+                    use_bits ^= 1u << k;
+                    const uint32_t pbuf = gbuf + (uint32_t)k * PART_BYTES;
+                    constexpr int CPP = PART_COLS / EPI_COLS;  // 32-column chunks per part
+                    for (int c = 0; c < CPP; ++c) {
                         uint32_t r[32];
-                        tc_ld_32x32(taddr0 + (uint32_t)(c * EPI_COLS), r);
+                        tc_ld_32x32(taddr0 + (uint32_t)((part_i * CPP + c) * EPI_COLS), r);
                         tc_wait_ld();
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
-                            st_shared_v4(gbuf + (uint32_t)lrow * 1024u +
+                            st_shared_v4(pbuf + (uint32_t)lrow * (PART_COLS * 4) +
                                              (uint32_t)(((c * 8 + j) ^ (lrow & 7)) << 4),
                                          __uint_as_float(r[4 * j + 0]), __uint_as_float(r[4 * j + 1]),
                                          __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars->g_full[h]));
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->g_full[k]));
                 }
                 if (!ok) break;
                 // the accumulator stage may be overwritten
@@ -1103,9 +1116,10 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
     // calls of few tokens: staged epilogue (see STAGED_RING)
-    // (4096x4096, L2 flushed, staged vs not: 256 tokens 65.6 vs 75.8 us, 1024 tokens 71.7 vs 79.9,
-    // 2048 tokens 92.1 vs 82.0 -- there the 3-stage ring starves the main loop)
-    const bool staged = g_force_staged ? g_force_staged > 0 : p.tokens <= 1024;
+    // (4096x4096, L2 flushed, staged vs direct epilogue, us: 256 tokens 65.6 vs 75.8, 1024: 69.7 vs
+    // 79.9, 2048: 75.8 vs 82.0, 3072: 94.2 vs 92.2, 4096: 114.7 vs 110.6.  With 128-column parts and
+    // the 3-stage ring they leave: 66.6, 71.7, 92.2 at 256, 1024, 2048 tokens.)
+    const bool staged = g_force_staged ? g_force_staged > 0 : p.tokens <= 2048;
     cfg.dynamicSmemBytes = staged ? Geo<2, true>::SMEM_BYTES : Geo<2>::SMEM_BYTES;
     if (staged) cfg.blockDim = dim3((unsigned)(STAGED_THREADS - (p.bias_m ? 0 : 32 * BIAS_WARPS)), 1, 1);
     cfg.stream = p.stream;

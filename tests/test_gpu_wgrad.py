@@ -114,12 +114,12 @@ def test_ragged_shapes(T, d_in, d_out):
     _full_parity(T, d_in, d_out, integer=True, pad=5)
 
 
-@pytest.mark.parametrize("T", [1030, 1100, 2100])
+@pytest.mark.parametrize("T", [1100, 2048, 2100, 2500])
 @pytest.mark.parametrize("d_in,d_out", [(200, 328), (129, 263), (136, 520), (300, 1000)])
-def test_ragged_shapes_beyond_the_short_call_path(T, d_in, d_out):
-    """Calls of up to 1024 tokens take the staged epilogue (accumulator -> shared memory ->
-    streaming fold); these token counts take the direct epilogue instead, on the same ragged
-    shapes and padded buffers.  Integer inputs: exact contraction, fp32 fold tolerance."""
+def test_ragged_shapes_on_both_sides_of_the_short_call_limit(T, d_in, d_out):
+    """Calls of up to 2048 tokens take the staged epilogue (accumulator -> shared memory ->
+    streaming fold), longer ones the direct epilogue; the same ragged shapes and padded buffers
+    on both sides of the limit.  Integer inputs: exact contraction, fp32 fold tolerance."""
     _full_parity(T, d_in, d_out, integer=True, pad=5)
 
 
