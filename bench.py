@@ -232,7 +232,7 @@ def run_ours(args):
 
     n = args.flat_params
     NA, NB = wl.CONFIG2.n_micro, wl.CONFIG3.n_micro
-    T, d_in, d_out = wl.CONFIG3.tokens, wl.CONFIG3.d_in, wl.CONFIG3.d_out
+    T, d_in, d_out = args.linear_tokens, wl.CONFIG3.d_in, wl.CONFIG3.d_out
     seed_shift = 100000 * rank  # each rank owns its own replica's data (weak scaling)
 
     # phase A state and inputs
@@ -910,6 +910,9 @@ def main():
     ap.add_argument("--biases", action="store_true",
                     help="gpt2xl workload: give every linear layer a bias, folded in the fused launch")
     ap.add_argument("--flat-params", type=int, default=wl.CONFIG2_FULL_N)
+    ap.add_argument("--linear-tokens", type=int, default=wl.CONFIG3.tokens,
+                    help="tokens per micro-batch of the linear layer (default: the workload's 4096; "
+                         "smaller values are for profiling the short-call kernel instance)")
     ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing", "wgrad_shapes"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
