@@ -25,6 +25,10 @@
 // The 512 TMEM columns hold two 128x256 fp32 accumulators per CTA, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  (A one-CTA variant, 128x256 tiles and a
 // 4-stage ring, is kept as a template instance for comparison.)
+//   optional    two more warps that sum dY's columns into the bias moments (see the bias branch)
+// Calls of up to 2048 tokens run a second instance with a "staged" epilogue (see STAGED_RING):
+// 4 drain warps copy the accumulator to shared memory part by part, 8 streaming warps fold
+// the parts into m and v; the ring has 5 stages there.
 //
 // Operand layout.  The contraction runs over tokens, the strided dimension of both
 // row-major inputs, so both operands are "MN-major": a TMA box of 64 features x 64
