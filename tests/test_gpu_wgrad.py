@@ -263,3 +263,35 @@ def test_host_buffer_variants_match_device_variants():
         opt.close()
     for a, b in zip(*res):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("T", [512, 4096])
+def test_inputs_written_just_before_the_call_and_overwritten_just_after(T):
+    """The fused kernel is launched so that its set-up may overlap the end of the kernel before
+    it in the stream.  Here that kernel is the one that WRITES dY (and X), and the next one
+    overwrites them again at once, 30 times over without any synchronisation: the result must be
+    bit-identical to the same sequence with a device synchronisation after every operation."""
+    d_in, d_out, rounds = 512, 768, 30
+    Xs = [wl.normal((T, d_in), 1.0, torch.bfloat16, 900 + i, device="cuda") for i in range(3)]
+    Ys = [wl.normal((T, d_out), 1e-2, torch.bfloat16, 950 + i, device="cuda") for i in range(3)]
+    outs = []
+    for sync in (True, False):
+        opt = adama.AdamA()
+        opt.begin_minibatch(rounds)
+        X = torch.zeros(T, d_in, dtype=torch.bfloat16, device="cuda")
+        dY = torch.zeros(T, d_out, dtype=torch.bfloat16, device="cuda")
+        m = torch.zeros(d_in, d_out, device="cuda")
+        v = torch.zeros(d_in, d_out, device="cuda")
+        for i in range(rounds):
+            X.copy_(Xs[i % 3])
+            dY.copy_(Ys[(i + 1) % 3])
+            if sync:
+                torch.cuda.synchronize()
+            opt.linear_wgrad_fold(X, dY, m, v)
+            if sync:
+                torch.cuda.synchronize()
+        opt.sync_status()
+        outs.append((m.clone(), v.clone()))
+        opt.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    assert float(outs[0][1].max()) > 0
