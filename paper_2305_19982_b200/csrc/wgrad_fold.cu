@@ -404,7 +404,11 @@ __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars,
 }
 
 // Work list of a launch.  Items [0, split_from) are full tiles (TILE_M x 256), numbered
-// with the row-tile index fastest.  Items from split_from on are the two 128-column halves
+// with the index of the SHORTER tile dimension fastest: the ~74 tiles that run at the same
+// time then span a nearly square block of the tile grid and share the fewest distinct operand
+// blocks in the L2 (11008 x 4096 is 43 x 16 tiles: 74 consecutive tiles touch 5 row blocks and
+// 16 column blocks with the column index fastest, 43 and 2 with the row index fastest).
+// Items from split_from on are the two 128-column halves
 // of the remaining full tiles: when the last round would occupy at most half of the CTA
 // groups, halving its tiles halves its duration (the token sum of each half is still
 // complete, so the square stays exact).
@@ -412,7 +416,7 @@ struct WorkItem {
     int m0, n0, width;
 };
 template <int CTAS>
-__device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m) {
+__device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m, int tiles_n) {
     int full = w, half = 0, width = BN;
     if (w >= split_from) {
         const int j = w - split_from;
@@ -420,7 +424,9 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
         half = j & 1;
         width = BN / 2;
     }
-    return {(full % tiles_m) * Geo<CTAS>::TILE_M, (full / tiles_m) * BN + half * (BN / 2), width};
+    const int tm = tiles_n < tiles_m ? full / tiles_n : full % tiles_m;
+    const int tn = tiles_n < tiles_m ? full % tiles_n : full / tiles_m;
+    return {tm * Geo<CTAS>::TILE_M, tn * BN + half * (BN / 2), width};
 }
 
 template <int CTAS, bool STAGED>
@@ -450,6 +456,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     const int group = blockIdx.x / CTAS;                           // which pair
     const int num_groups = gridDim.x / CTAS;
     const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
+    const int tiles_n = (d_out + BN - 1) / BN;
     const int num_kb = (tokens + BK - 1) / BK;
     // warps 2 .. 2+epi_warps-1: epilogue; with bias moments, BIAS_WARPS more after them
     // (staged: 4 drain warps take the epilogue's place, 8 streaming warps follow them)
@@ -500,7 +507,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             // the pair's loads are counted by the first CTA's barrier
             const uint32_t full0_lead = (CTAS == 1) ? full0 : map_to_cta(full0, 0);
             for (int tile = group; tile < num_items && ok; tile += num_groups) {
-                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
                 const int cols_per_cta = wi.width / CTAS;  // dY columns this CTA stages
                 const int b_boxes = cols_per_cta / GROUP;
                 const int m0 = wi.m0 + (int)rank * G::ROWS_PER_CTA;
@@ -573,7 +580,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
                 const uint32_t idesc =
                     G::INSTR_DESC_NO_N |
-                    ((uint32_t)(work_item<CTAS>(tile, split_from, tiles_m).width >> 3) << 17);
+                    ((uint32_t)(work_item<CTAS>(tile, split_from, tiles_m, tiles_n).width >> 3) << 17);
                 ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
                 if (!ok) {
                     record_timeout(status, bars, 2, (unsigned)tile);
@@ -647,7 +654,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         uint32_t use_bits = 0;    // bit k: parity of how often part buffer k has been used
         grid_dependency_wait();   // m and v may still be written by the previous call
         for (int tile = group; tile < num_items && ok; tile += num_groups) {
-            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
             const int row_base = wi.m0 + (int)rank * G::ROWS_PER_CTA;
             for (int part_i = 0; part_i < wi.width / PART_COLS; ++part_i) {
                 if (!ok) continue;
@@ -808,7 +815,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
                 ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) {
@@ -874,7 +881,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m);
+            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
             const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
             const int chunks = wi.width / (col_split * EPI_COLS);  // chunks per warp
             ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
