@@ -65,6 +65,15 @@ def load_library() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
+    if not _LIB_PATH.exists() and _LIB_PATH == _PKG / "libadama.so":
+        # a source-only checkout: compile once, in-tree (needs nvcc); never a substitute path
+        try:
+            from . import build as _build
+            _build.build()
+        except Exception as exc:  # noqa: BLE001 - reported below with the way out
+            raise FileNotFoundError(
+                f"{_LIB_PATH} is missing and could not be built ({exc}): build it with "
+                "`python -m paper_2305_19982_b200.build` (there is no fallback path)") from exc
     if not _LIB_PATH.exists():
         raise FileNotFoundError(
             f"{_LIB_PATH} is missing: build it with `python -m paper_2305_19982_b200.build` "
