@@ -101,4 +101,4 @@ def llama7b_block_linears() -> List[Tuple[str, int, int]]:
 
 
 CONFIG4_BLOCKS, CONFIG4_TOKENS, CONFIG4_N_MICRO = 48, 4 * 1024, 8
-CONFIG5_BLOCKS, CONFIG5_TOKENS, CONFIG5_N_MICRO = 32, 4096, 16
+CONFIG5_BLOCKS, CONFIG5_TOKENS, CONFIG5_N_MICRO, CONFIG5_STEPS = 32, 4096, 16, 2

@@ -157,21 +157,30 @@ def make_oracle_state(n_flat, tokens, d_in, d_out):
             "threads": oracle.num_threads()}
 
 
-def time_oracle(n_flat, tokens, d_in, d_out, steps, warmup):
+# The bounded sample of the headline step that the oracle is timed on, in BOTH arms (the
+# cpu_baseline of the default run and --impl reference): flat 2^24 parameters, linear layer
+# 512 x 512 with 256 tokens.
+ORACLE_SAMPLE = (1 << 24, 256, 512, 512)
+
+
+def time_oracle(n_flat, tokens, d_in, d_out, steps, warmup, min_seconds=0.0):
+    """Times `steps` sample steps (more, up to 50x, until `min_seconds` of work have run)."""
     state = make_oracle_state(n_flat, tokens, d_in, d_out)
     for _ in range(warmup):
         oracle_sample_step(state)
     t0 = time.perf_counter()
-    for _ in range(steps):
+    done = 0
+    while done < steps or (time.perf_counter() - t0 < min_seconds and done < 50 * steps):
         oracle_sample_step(state)
-    dt = (time.perf_counter() - t0) / steps
+        done += 1
+    dt = (time.perf_counter() - t0) / done
     flat_b, lin_b, flops, _ = step_bytes_and_flops(n_flat, wl.CONFIG2.n_micro, tokens, d_in, d_out,
                                                    wl.CONFIG3.n_micro)
     sample = (f"flat buffer of {n_flat} params (of {wl.CONFIG2_FULL_N}), N=8 bf16-valued grads; "
               f"linear layer {d_in}x{d_out}, {tokens} tokens (of 4096x4096, 4096), N=4; "
               "same flow, fp64, OpenMP over elements")
     return {"value": (flat_b + lin_b) / dt / 1e9, "unit": UNIT, "cores": state["threads"],
-            "kind": "oracle", "sample": sample, "seconds_per_sample_step": dt,
+            "kind": "oracle", "sample": sample, "seconds_per_sample_step": dt, "sample_steps": done,
             "wgrad_gflops": flops / dt / 1e9}
 
 
@@ -179,7 +188,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    base = time_oracle(1 << 24, 256, 512, 512, args.steps, args.warmup)
+    base = time_oracle(*ORACLE_SAMPLE, args.steps, args.warmup)
     line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": base["seconds_per_sample_step"] * 1e3, "higher_is_better": True,
@@ -252,20 +261,45 @@ def run_ours(args):
     dYs = [wl.normal((T, d_out), 1e-2, torch.bfloat16, wl.seed_for(3, 0, i) + 50 + seed_shift,
                      device=dev) for i in range(NB)]
 
+    # Data-parallel exchange at the end of each mini-batch (Section 3.3: the STATES are reduced,
+    # once per mini-batch): "none" = independent replicas; "allreduce" = all-reduce of m and v,
+    # then the update with the 1/R, 1/R^2 of Eqs. 6-7 folded in; "sharded" = reduce-scatter of
+    # m and v, update of the owner's shard, all-gather of w.
+    exchange = args.exchange if world > 1 else "none"
+    if exchange != "none":
+        from paper_2305_19982_b200 import ddp
+    if exchange == "sharded" and (n % world or (d_in * d_out) % world):
+        raise SystemExit("--exchange sharded needs buffer lengths that are multiples of the world size")
+
+    def finish(opt, w_, m_, v_, label):
+        if exchange == "allreduce":
+            mark_ex(label + "_exchange")
+            ddp.allreduce_states(m_, v_)
+            mark_ex(label)
+            opt.apply_allreduced(w_, m_, v_, wl.LR, world)
+        elif exchange == "sharded":
+            mark_ex(label + "_exchange")
+            ddp.reduce_scatter_apply_allgather(opt, w_, m_, v_, wl.LR)
+        else:
+            mark_ex(label)
+            opt.apply(w_, m_, v_, wl.LR)
+
+    mark_ex = lambda label: None
+
     def step(timer=None):
+        nonlocal mark_ex
         mark = timer.mark if timer else (lambda label: None)
+        mark_ex = mark
         optA.begin_minibatch(NA)
         for i in range(NA):
             mark("fold")
             optA.fold(grads[i], m, v)
-        mark("apply")
-        optA.apply(w, m, v, wl.LR)
+        finish(optA, w, m, v, "apply")
         optB.begin_minibatch(NB)
         for i in range(NB):
             mark("wgrad_fold")
             optB.linear_wgrad_fold(Xs[i], dYs[i], mB, vB)
-        mark("apply_linear")
-        optB.apply(wB, mB, vB, wl.LR)
+        finish(optB, wB, mB, vB, "apply_linear")
         mark(None)
 
     def barrier():
@@ -306,7 +340,10 @@ def run_ours(args):
     dur = timer.durations()
     avg = {k: sum(x) / len(x) for k, x in dur.items()}
     fold_gbs = FOLD_BYTES_BF16 * n / (avg["fold"] * 1e-3) / 1e9
-    apply_gbs = APPLY_BYTES * n / (avg["apply"] * 1e-3) / 1e9
+    # (with --exchange sharded the update runs inside the exchange helper: no separate figure)
+    apply_gbs = APPLY_BYTES * n / (avg["apply"] * 1e-3) / 1e9 if "apply" in avg else 0.0
+    avg.setdefault("apply", 0.0)
+    dur.setdefault("apply", [0.0])
     wgrad_tf = 2.0 * T * d_in * d_out / (avg["wgrad_fold"] * 1e-3) / 1e12
     roof_kernels = {
         "fold_bf16": {"bound": "hbm", "achieved": fold_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
@@ -322,13 +359,15 @@ def run_ours(args):
                        "hbm_bytes_per_call": lin_call_b, "traffic": None,
                        "hbm_gbs": lin_call_b / (avg["wgrad_fold"] * 1e-3) / 1e9},
     }
-    traffic = load_traffic()
+    traffic = load_traffic(n, T, d_in, d_out)
     for key in roof_kernels:
-        roof_kernels[key]["traffic"] = traffic.get(key)
+        roof_kernels[key]["traffic"] = traffic.get(key, {}).get("bytes_per_launch")
+        roof_kernels[key]["traffic_note"] = traffic.get(key, {}).get("note")
     roofline = {"kernel": "fold_vec_kernel<bf16> (dominant: 8 launches per step)",
                 "bound": "hbm", "achieved": fold_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": fold_gbs / pk["hbm_gbs"], "peak_source": pk["source"],
-                "traffic": traffic.get("fold_bf16")}
+                "traffic": traffic.get("fold_bf16", {}).get("bytes_per_launch"),
+                "traffic_note": traffic.get("fold_bf16", {}).get("note")}
 
     # ---- end to end through the host-buffer entry points --------------------------------------
     e2e = None
@@ -336,14 +375,45 @@ def run_ours(args):
         e2e = run_e2e(adama, dev, local, n, NA, NB, T, d_in, d_out, w, m, v, wB, mB, vB,
                       max(1, min(args.steps, 10)), flat_b + lin_b, world, dist)
 
+    if "NCCL_DEBUG" in os.environ and rank == 0 and world > 1:
+        sys.stderr.write(f"[bench] NCCL_DEBUG={os.environ['NCCL_DEBUG']}: communicator log above\n")
+
+    # bytes each rank sends (= receives) per step in the exchange: ring all-reduce 2(R-1)/R of
+    # the payload, reduce-scatter and all-gather (R-1)/R each
+    params = n + d_in * d_out
+    exchange_info = {"mode": exchange, "bytes_per_rank_per_step": 0}
+    if exchange == "allreduce":
+        exchange_info["bytes_per_rank_per_step"] = int(2 * (world - 1) / world * 8 * params)
+        exchange_info["payload"] = "m and v, fp32 (8 B/param), one all-reduce each per mini-batch"
+    elif exchange == "sharded":
+        exchange_info["bytes_per_rank_per_step"] = int((world - 1) / world * 12 * params)
+        exchange_info["payload"] = "reduce-scatter of m, v (8 B/param) + all-gather of w (4 B/param)"
+    if exchange != "none":
+        exchange_info["ms_per_step"] = (sum(dur.get("apply_exchange", [0.0])) +
+                                        sum(dur.get("apply_linear_exchange", [0.0]))) / args.steps
+
     cpu_base = None
     peak_mem = None
+    stacks = None
     if rank == 0:
         peak_mem = memory_report(adama, dev, local, T, d_in, d_out, Xs[0], dYs[0])
+    optA.close()
+    optB.close()
+    del w, m, v, grads, wB, mB, vB, Xs, dYs
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_stacks:
+        # the two layer-stack workloads in their stated configuration, 2 mini-batches each
+        stacks = {"gpt2xl": measure_stack("gpt2xl", 2, 1, dev_index=local)}
+        free, _ = torch.cuda.mem_get_info()
+        if free >= 100 * (1 << 30):
+            stacks["llama7b"] = measure_stack("llama7b", 2, 1, dev_index=local)
+        else:
+            stacks["llama7b"] = {"skipped": f"needs ~90 GB of free device memory, {free >> 30} GiB free"}
+    if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            cpu_base = time_oracle(1 << 25, 512, 512, 1024, 2, 1)
+            cpu_base = time_oracle(*ORACLE_SAMPLE, 2, 1, min_seconds=10.0)
             cpu_base = {k: cpu_base[k] for k in ("value", "unit", "cores", "kind", "sample",
-                                                 "seconds_per_sample_step")}
+                                                 "seconds_per_sample_step", "sample_steps")}
 
     if rank == 0:
         line = {
@@ -354,24 +424,27 @@ def run_ours(args):
             "config": {"workload": f"headline: flat {n}-param buffer (bf16 grads, N={NA}) fold+apply, "
                                    f"then linear {d_in}x{d_out} with {T} tokens (N={NB}) fused "
                                    "wgrad+fold + apply",
-                       "l2": "inputs larger than L2, no flush", "replicas": world},
+                       "l2": "inputs larger than L2, no flush", "replicas": world,
+                       "exchange": exchange_info},
             "fold_apply_GBps": (flat_b / ((sum(dur["fold"]) + sum(dur["apply"])) / args.steps * 1e-3)) / 1e9,
             "wgrad_fold_TFLOPps": wgrad_tf,
             "roofline": roofline, "roofline_kernels": roof_kernels,
             "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks, "peak_memory": peak_mem,
+            "clocks": clocks, "peak_memory": peak_mem, "stacks": stacks,
         }
         print(json.dumps(line), flush=True)
-    optA.close()
-    optB.close()
     if dist is not None:
         dist.barrier()  # rank 0 may still be printing; leave the group together
         dist.destroy_process_group()
 
 
-def load_traffic():
-    """Per-launch DRAM traffic (bytes) from the committed ncu summaries, keyed by kernel; an
-    entry counts only while the kernel's source files are the ones the counters were taken on."""
+def load_traffic(n_flat, tokens, d_in, d_out):
+    """Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the committed
+    ncu summaries, scaled to THIS run's launch.  The streaming kernels were captured on a
+    smaller buffer (their traffic is proportional to the element count); the figure is a lower
+    bound, because the last stores of the small captured launch were still in the L2 when it
+    ended.  The fused call's entry counts only for the shape it was captured on.  An entry is
+    dropped once one of the kernel's source files differs from those the counters were taken on."""
     import hashlib
     p = ROOT / "profiles" / "traffic.json"
     out = {}
@@ -390,8 +463,17 @@ def load_traffic():
         h = hashlib.sha256()
         for f in srcs:
             h.update(f.read_bytes())
-        if h.hexdigest() == ent.get("sha256"):
-            out[key] = ent.get("bytes_per_launch")
+        if h.hexdigest() != ent.get("sha256"):
+            continue
+        if "captured_params" in ent:
+            scale = n_flat / ent["captured_params"]
+            out[key] = {"bytes_per_launch": int(ent["captured_bytes"] * scale),
+                        "note": f"scaled from a {ent['captured_params']}-param capture "
+                                f"({ent['captured_bytes'] / ent['captured_params']:.2f} B/param); lower "
+                                "bound (stores still in the L2 when the captured launch ended)"}
+        elif ent.get("shape") == [tokens, d_in, d_out]:
+            out[key] = {"bytes_per_launch": int(ent["captured_bytes"]),
+                        "note": "captured on this shape"}
     return out
 
 
@@ -480,23 +562,41 @@ def memory_report(adama, dev, local, T, d_in, d_out, X, dY):
             "note": "bytes above the resident state and inputs during one micro-batch of the layer"}
 
 
-def run_stack(args):
-    """GPT-2-XL- / Llama-7B-shaped stacks: one mini-batch per step, layers back to front,
-    fused weight-gradient fold per layer, one apply; reports TFLOP/s of the whole mini-batch
-    and peak device memory with and without materialised gradients."""
+def materialised_minibatch(stack, opt, n_micro, lr, inputs):
+    """Comparison arm only, never the product path: the paper's own pipeline, in which every
+    layer's fp32 weight gradient is assigned a buffer, filled by a library GEMM (cuBLAS through
+    torch.mm), folded with adama_fold and released."""
+    opt.begin_minibatch(n_micro)
+    for i in range(n_micro):
+        for j in reversed(range(len(stack.layers))):
+            spec = stack.layers[j]
+            X, dY = inputs(i, j, spec)
+            G = torch.empty(spec.d_in, spec.d_out, dtype=torch.float32, device=stack.device)
+            torch.mm(X.t(), dY, out_dtype=torch.float32, out=G)
+            opt.fold(G.view(-1), stack.view(stack.m, j).view(-1), stack.view(stack.v, j).view(-1))
+            del G
+            if stack.biases:
+                opt.bias_grad_fold(dY, stack.bias_view(stack.m, j), stack.bias_view(stack.v, j))
+            del X, dY
+    stack.apply(opt, lr)
+
+
+def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, dev_index=0):
+    """GPT-2-XL- / Llama-7B-shaped stack, one mini-batch per step in the workload's own
+    configuration (N = 8 / 16 micro-batches of 4096 tokens, layers back to front, fused
+    weight-gradient fold per layer, one apply): time, TFLOP/s of the whole mini-batch, clocks,
+    peak device memory without a gradient buffer, with a per-layer one and with a whole-model one."""
     import paper_2305_19982_b200 as adama
     from paper_2305_19982_b200.stack import gpt2xl_stack, llama7b_stack
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
+    dev = torch.device("cuda", dev_index)
     pk = peaks()
-    if args.workload == "gpt2xl":
-        stack, tokens, n_micro, cfg_id = (gpt2xl_stack(wl.CONFIG4_BLOCKS, biases=args.biases), wl.CONFIG4_TOKENS,
-                                          wl.CONFIG4_N_MICRO, 4)
+    if kind == "gpt2xl":
+        stack, tokens, n_micro, cfg_id = (gpt2xl_stack(wl.CONFIG4_BLOCKS, device=dev, biases=biases),
+                                          wl.CONFIG4_TOKENS, wl.CONFIG4_N_MICRO, 4)
     else:
-        stack, tokens, n_micro, cfg_id = llama7b_stack(wl.CONFIG5_BLOCKS), wl.CONFIG5_TOKENS, wl.CONFIG5_N_MICRO, 5
+        stack, tokens, n_micro, cfg_id = (llama7b_stack(wl.CONFIG5_BLOCKS, device=dev),
+                                          wl.CONFIG5_TOKENS, wl.CONFIG5_N_MICRO, 5)
     stack.w.normal_(0, 0.02, generator=torch.Generator(device=dev).manual_seed(wl.seed_for(cfg_id, 99)))
     # two seeded variants of X and dY per distinct width, reused across layers while timing
     widths = sorted({L.d_in for L in stack.layers} | {L.d_out for L in stack.layers})
@@ -504,43 +604,42 @@ def run_stack(args):
                   for k in range(2)] for d in widths}
     pool_y = {d: [wl.normal((tokens, d), 1e-2, torch.bfloat16, wl.seed_for(cfg_id, 0, k) + 50 + d, device=dev)
                   for k in range(2)] for d in widths}
-    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
+    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=dev_index)
 
     def pooled(i, j, spec):
         return pool_x[spec.d_in][(i + j) & 1], pool_y[spec.d_out][(i + j) & 1]
 
-    def step(mode="none"):
-        stack.minibatch(opt, n_micro, wl.LR, pooled, materialise=mode)
-
-    for _ in range(max(1, min(args.warmup, 2))):
-        step()
+    for _ in range(max(1, warmup)):
+        stack.minibatch(opt, n_micro, wl.LR, pooled)
     torch.cuda.synchronize()
-    sampler = ClockSampler(physical_gpu_index(0))
+    sampler = ClockSampler(physical_gpu_index(dev_index))
     sampler.start()
     launches0 = opt.launch_count
     start = torch.cuda.Event(enable_timing=True)
     stop = torch.cuda.Event(enable_timing=True)
     start.record()
-    for _ in range(args.steps):
-        step()
+    for _ in range(steps):
+        stack.minibatch(opt, n_micro, wl.LR, pooled)
     stop.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    ms = start.elapsed_time(stop) / args.steps
+    ms = start.elapsed_time(stop) / steps
     launches = opt.launch_count - launches0
     opt.sync_status()
     flops = n_micro * stack.flops_per_micro_batch(tokens)
     tf = flops / (ms * 1e-3) / 1e12
-    # the paper's pipeline (per-layer gradient assigned, folded, released) for comparison
-    step("layer")
-    torch.cuda.synchronize()
-    s2 = torch.cuda.Event(enable_timing=True)
-    e2 = torch.cuda.Event(enable_timing=True)
-    s2.record()
-    step("layer")
-    e2.record()
-    torch.cuda.synchronize()
-    ms_layer = s2.elapsed_time(e2)
+    ms_layer = None
+    if with_gemm_pipeline:
+        # the paper's pipeline (per-layer gradient assigned, folded, released) for comparison
+        materialised_minibatch(stack, opt, n_micro, wl.LR, pooled)
+        torch.cuda.synchronize()
+        s2 = torch.cuda.Event(enable_timing=True)
+        e2 = torch.cuda.Event(enable_timing=True)
+        s2.record()
+        materialised_minibatch(stack, opt, n_micro, wl.LR, pooled)
+        e2.record()
+        torch.cuda.synchronize()
+        ms_layer = s2.elapsed_time(e2)
 
     # peak memory: fresh X, dY per layer (as a backward pass would hand them over)
     def fresh(i, j, spec):
@@ -553,26 +652,23 @@ def run_stack(args):
     for mode in ("none", "layer"):
         torch.cuda.synchronize()
         torch.cuda.reset_peak_memory_stats(dev)
-        stack.minibatch(opt, 1, wl.LR, fresh, materialise=mode)
+        if mode == "none":
+            stack.minibatch(opt, 1, wl.LR, fresh)
+        else:
+            materialised_minibatch(stack, opt, 1, wl.LR, fresh)
         torch.cuda.synchronize()
         mem[mode] = int(torch.cuda.max_memory_allocated(dev))
+    opt.sync_status()
     state_bytes = 3 * 4 * stack.numel
     largest_layer = max(L.d_in * L.d_out for L in stack.layers)
-    line = {
-        "metric": "adama_wgrad_fold_stack_TFLOPps", "value": tf, "unit": "TFLOP/s", "n_gpus": 1,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate and state",
-        "data": "synthetic",
-        "config": {"workload": args.workload, "biases": bool(getattr(stack, "biases", False)),
-                   "layers": len(stack.layers), "params": stack.n_params,
-                   "tokens_per_micro_batch": tokens, "n_micro": n_micro,
-                   "l2": "inputs larger than L2, no flush"},
-        "roofline": {"kernel": "wgrad_fold_kernel<2>", "bound": "tensor", "achieved": tf,
-                     "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": tf / pk["bf16_tflops_sustained"],
-                     "frac_of_burst": tf / pk["bf16_tflops"], "peak_source": pk["source"] + " (sustained)",
-                     "traffic": None},
-        "materialised_per_layer_ms_per_step": ms_layer,
+    out = {
+        "workload": kind, "biases": bool(stack.biases), "layers": len(stack.layers),
+        "params": stack.n_params, "tokens_per_micro_batch": tokens, "n_micro": n_micro,
+        "steps": steps, "ms_per_minibatch": ms, "TFLOPps": tf,
+        "frac_of_sustained_bf16": tf / pk["bf16_tflops_sustained"],
+        "frac_of_burst_bf16": tf / pk["bf16_tflops"], "peak_source": pk["source"],
+        "gpu_launches": int(launches), "clocks": clocks,
+        "gemm_plus_fold_pipeline_ms_per_minibatch": ms_layer,
         "peak_memory": {"state_bytes": state_bytes,
                         "fused_no_gradient_buffer": mem["none"],
                         "per_layer_gradient_released": mem["layer"],
@@ -580,10 +676,37 @@ def run_stack(args):
                         "largest_layer_gradient_bytes": 4 * largest_layer,
                         "note": "max_memory_allocated over one micro-batch with fresh X, dY per layer; "
                                 "the gradient-accumulation figure adds an fp32 gradient for every parameter"},
-        "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+    }
+    opt.close()
+    del stack
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_stack(args):
+    """One stack workload on its own (python bench.py --workload gpt2xl|llama7b)."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    r = measure_stack(args.workload, args.steps, min(args.warmup, 2), biases=args.biases)
+    pk = peaks()
+    line = {
+        "metric": "adama_wgrad_fold_stack_TFLOPps", "value": r["TFLOPps"], "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_minibatch"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 inputs, f32 accumulate and state", "data": "synthetic",
+        "config": {"workload": args.workload, "biases": r["biases"], "layers": r["layers"],
+                   "params": r["params"], "tokens_per_micro_batch": r["tokens_per_micro_batch"],
+                   "n_micro": r["n_micro"], "l2": "inputs larger than L2, no flush"},
+        "roofline": {"kernel": "wgrad_fold_kernel", "bound": "tensor", "achieved": r["TFLOPps"],
+                     "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": r["frac_of_sustained_bf16"], "frac_of_burst": r["frac_of_burst_bf16"],
+                     "peak_source": pk["source"] + " (sustained)", "traffic": None},
+        "materialised_per_layer_ms_per_step": r["gemm_plus_fold_pipeline_ms_per_minibatch"],
+        "peak_memory": r["peak_memory"],
+        "cpu_baseline": None, "e2e": None, "gpu_launches": r["gpu_launches"], "clocks": r["clocks"],
     }
     print(json.dumps(line), flush=True)
-    opt.close()
 
 
 def run_sweep(args):
@@ -901,6 +1024,46 @@ def run_small_tensors(args):
     opt.close()
 
 
+def run_launch_check(args):
+    """The multi-rank plumbing of the benchmark without any GPU work (used by the CPU tests with
+    the gloo backend): rendezvous, barrier, a timed no-op region, max over ranks, one line."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group(args.backend)
+        dist.barrier()
+    t0 = time.perf_counter()
+    time.sleep(0.01 * (rank + 1))
+    t = torch.tensor([(time.perf_counter() - t0) * 1e3], dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({"metric": "launch_check", "value": None, "n_gpus": world,
+                          "ms_per_step": float(t.item()), "gpu_launches": 0,
+                          "config": {"workload": "launch_check", "backend": args.backend}}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def relaunch_with_ranks(args):
+    """`python bench.py --gpus N` started without a launcher: start the N ranks here, one per
+    GPU, the way torchrun would (rendezvous on 127.0.0.1), and hand on their exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ)
+    # NCCL's communicator log (rings/trees, NVLS availability) goes to stderr with the run
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+           f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port", str(port),
+           str(Path(__file__).resolve())] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -913,12 +1076,24 @@ def main():
     ap.add_argument("--linear-tokens", type=int, default=wl.CONFIG3.tokens,
                     help="tokens per micro-batch of the linear layer (default: the workload's 4096; "
                          "smaller values are for profiling the short-call kernel instance)")
-    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing", "wgrad_shapes"])
+    ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing", "wgrad_shapes", "launch_check"])
+    ap.add_argument("--exchange", default="none", choices=["none", "allreduce", "sharded"],
+                    help="N > 1: what the ranks exchange at the end of each mini-batch, inside the "
+                         "timed step (none = independent replicas; allreduce = Section 3.3's state "
+                         "all-reduce; sharded = reduce-scatter of the states, all-gather of the weights)")
+    ap.add_argument("--backend", default="gloo", help="launch_check only: process-group backend")
+    ap.add_argument("--no-stacks", action="store_true",
+                    help="skip the two layer-stack workloads of the default line (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if (args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours"
+            and args.workload in ("headline", "launch_check")):
+        sys.exit(relaunch_with_ranks(args))
+    if args.workload == "launch_check":
+        run_launch_check(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.workload == "sweep":
         run_sweep(args)

@@ -120,9 +120,10 @@ ADAMA_API adama_status adama_fold(adama_ctx *ctx, const void *grad, adama_dtype 
                                   float *v, size_t n, void *cuda_stream);
 
 /* The same accumulation for a linear layer y = x.W, W of shape [d_in, d_out],
- * whose raw weight gradient is G = X^T.dY ("once the gradients of a layer are
- * produced" in Section 3.1; Algorithm 2's "assign / release memory for g"
- * disappears because G only ever exists as a tensor-memory accumulator tile):
+ * whose raw weight gradient is G = X^T.dY (Section 3.1 folds a layer's gradient
+ * into the moments as soon as backward has produced it; the buffer that Algorithm 2
+ * assigns and releases for it disappears because G only ever exists as a
+ * tensor-memory accumulator tile):
  *     G[p,q] = sum_{tau < tokens} X[tau,p] * dY[tau,q]   (bf16 x bf16 -> fp32)
  *     m[p,q] += a*G[p,q],   v[p,q] += b*G[p,q]^2
  *   X    : [tokens, d_in]  bf16 row-major, row pitch ldx  elements, device, read-only
@@ -148,10 +149,11 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
 
 /* adama_linear_wgrad_fold that also folds the layer's bias gradient, the column sums of dY,
  *     g[q] = sum_{tau < tokens} dY[tau,q],   m_bias[q] += a*g[q],   v_bias[q] += b*g[q]^2
- * (Algorithm 2, inner loop body, for the bias of the same layer) in the same launch: the
- * kernel's epilogue warps, idle until the first accumulator tile is complete, form the sums
- * meanwhile; every 32-column slab is summed over all tokens by one CTA, so the sum is
- * complete before it is squared, and the result is deterministic.
+ * (Algorithm 2, inner loop body, for the bias of the same layer) in the same launch: two
+ * extra warps per CTA read dY from global memory (it is L2-resident: the producer is loading
+ * the same data) and form the sums while the other roles run the tiles; every 32-column slab
+ * is summed over all tokens by one CTA, so the sum is complete before it is squared, and the
+ * result is deterministic.
  *   m_bias, v_bias : d_out fp32 elements each, contiguous, device, updated in place.
  * Weight results are bit-identical to adama_linear_wgrad_fold; the bias results equal
  * adama_bias_grad_fold's up to the order of the fp32 token sum.
@@ -216,7 +218,7 @@ ADAMA_API adama_status adama_apply_multi(adama_ctx *ctx, float *const *w, float 
  * stream order); this call then takes the summed buffers and computes
  *     m_t = m/R,  v_t = v/R^2                          (the paper's averaging of the states)
  *     w <- w - lr * (m_t/(1-beta1^t)) / (sqrt(v_t/(1-beta2^t)) + eps)
- *     m <- beta1*m_t,  v <- R*beta2*v_t                ("multiply v by M*beta2 instead of beta2")
+ *     m <- beta1*m_t,  v <- R*beta2*v_t                (Section 3.3: v decays by devices*beta2, Eq. 5)
  * so that R devices x N micro-batches give exactly the update of one device with N*R
  * micro-batches.  Every rank calls it with the same arguments and ends with the same w.
  * Between mini-batches each rank's v therefore holds R*beta2*v_t (m holds beta1*m_t).
@@ -401,6 +403,39 @@ ADAMA_API adama_status adama_sync_status(adama_ctx *ctx, void *cuda_stream);
  * any kernel wait in vain.  Synchronises `cuda_stream`. */
 ADAMA_API adama_status adama_debug_set_status(adama_ctx *ctx, unsigned code, unsigned wait,
                                               unsigned tile, void *cuda_stream);
+
+/* Test hook: makes a device-side wait of the fused weight-gradient kernel actually run out, in
+ * the non-hanging form.  Launches the kernel of adama_linear_wgrad_fold (same arguments, same
+ * checks) with every bounded wait limited to `wait_limit_ns` (>= 1000, <= 10^9) instead of
+ * 2 s, and with the producer told not to load the last 64-token stage of the launch's last
+ * tile.  The issuer's wait for that stage expires; it records {time-out, which wait, tile} in
+ * the status block, every role of the CTA pair gives up within its own limit, issued MMAs and
+ * loads are waited for, tensor memory is released and the kernel returns.  All other tiles of
+ * the launch are folded normally; the last tile's m, v are left untouched.  The following
+ * adama_sync_status returns ADAMA_ERR_TIMEOUT and clears the block; the context stays usable.
+ * No wait in the kernel is unbounded and nothing faults.  Errors: as adama_linear_wgrad_fold,
+ * plus INVALID_ARG for a limit out of range or tokens == 0. */
+ADAMA_API adama_status adama_debug_wgrad_expire_wait(adama_ctx *ctx, const void *X, const void *dY,
+                                                     int tokens, int d_in, int d_out, int64_t ldx,
+                                                     int64_t ldy, float *m, float *v, int64_t ldmv,
+                                                     uint64_t wait_limit_ns, void *cuda_stream);
+
+/* Test hook: pins which instance of the fused weight-gradient kernel this context launches, so
+ * that every instance can be checked on every shape whatever the automatic choice would be.
+ * 0 = automatic (the default).  epilogue: 1 = direct, 2 = staged through shared memory;
+ * epi_warps: 4 or 8 (direct epilogue); box_loads: 1 = one TMA operation per 64-feature box
+ * even where grouped loads apply; no_pdl: 1 = plain stream order instead of programmatic
+ * dependent launch; tile_cols: width of the column tiles (a multiple of 32 up to 256).
+ * Results do not depend on the choice beyond fp32 summation order inside the tensor cores
+ * (none: the order over tokens is the same).  Errors: INVALID_ARG for any other value. */
+ADAMA_API adama_status adama_debug_set_wgrad_variant(adama_ctx *ctx, int epilogue, int epi_warps,
+                                                     int box_loads, int no_pdl, int tile_cols);
+
+/* Diagnostics of the library's one-time set-up: bit 0 = the driver's tensor-map encoder has been
+ * resolved (once per process), bit 1 = the fused kernel's attributes have been set on `device`
+ * (once per device: a process that uses several GPUs sets each of them up at its first launch
+ * there).  Needs no GPU. */
+ADAMA_API int adama_debug_setup_state(int device);
 
 /* Message for the most recent non-OK status returned on this context ("" if
  * none).  The pointer stays valid until the next call on the context. */

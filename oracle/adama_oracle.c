@@ -178,8 +178,8 @@ ORACLE_API void oracle_linear_wgrad_entries(const double *X, const double *dY, i
 }
 
 /* Section 3.3, data-parallel variant, start of a mini-batch on one device:
- * "multiply v_{t-1} by M*beta2 instead of beta2" (M = number of devices);
- * m is decayed by beta1 as before (Eqs. 4-5). */
+ * v_{t-1} is scaled by devices*beta2 where the single-device algorithm scales it
+ * by beta2; m is decayed by beta1 as before (Eqs. 4-5). */
 ORACLE_API void oracle_ddp_decay(double *m, double *v, size_t n, int devices,
                                  double beta1, double beta2) {
 #pragma omp parallel for schedule(static)

@@ -7,7 +7,7 @@ stream).  There is no CPU fallback: importing works without a GPU, but creating
 an ``AdamA`` context raises if the library or a sm_100 device is missing.
 """
 from .binding import (AdamA, AdamAError, TensorList, Status, library_path, load_library, host_constants,
-                      linear_wgrad_fold_noalloc, EXPORTED_SYMBOLS)
+                      linear_wgrad_fold_noalloc, debug_setup_state, EXPORTED_SYMBOLS)
 
 __all__ = ["AdamA", "AdamAError", "TensorList", "Status", "library_path", "load_library", "host_constants",
-           "linear_wgrad_fold_noalloc", "EXPORTED_SYMBOLS"]
+           "linear_wgrad_fold_noalloc", "debug_setup_state", "EXPORTED_SYMBOLS"]

@@ -21,7 +21,8 @@ EXPORTED_SYMBOLS = [
     "adama_fold_host", "adama_linear_wgrad_fold_host",
     "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_sgdm_fold", "adama_sgdm_apply",
     "adama_coefficient_stats", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
-    "adama_sync_status", "adama_debug_set_status", "adama_last_error", "adama_launch_count", "adama_host_constants",
+    "adama_sync_status", "adama_debug_set_status", "adama_debug_wgrad_expire_wait",
+    "adama_debug_set_wgrad_variant", "adama_debug_setup_state", "adama_last_error", "adama_launch_count", "adama_host_constants",
     "adama_host_constants_allreduced", "adama_host_constants_sharded",
     "adama_version",
 ]
@@ -115,6 +116,11 @@ def load_library() -> ctypes.CDLL:
     L.adama_set_weight_decay.argtypes = [vp, dbl]
     L.adama_sync_status.argtypes = [vp, vp]
     L.adama_debug_set_status.argtypes = [vp, ctypes.c_uint, ctypes.c_uint, ctypes.c_uint, vp]
+    L.adama_debug_wgrad_expire_wait.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64,
+                                                ctypes.c_uint64, vp]
+    L.adama_debug_set_wgrad_variant.argtypes = [vp, ci, ci, ci, ci, ci]
+    L.adama_debug_setup_state.argtypes = [ci]
+    L.adama_debug_setup_state.restype = ci
     L.adama_last_error.argtypes = [vp]
     L.adama_last_error.restype = ctypes.c_char_p
     L.adama_launch_count.argtypes = [vp]
@@ -487,6 +493,24 @@ class AdamA:
         self._check(self._L.adama_debug_set_status(self._h, code, wait, tile,
                                                    _stream_ptr(self.device)))
 
+    def debug_wgrad_expire_wait(self, X: torch.Tensor, dY: torch.Tensor, m: torch.Tensor,
+                                v: torch.Tensor, wait_limit_ns: int) -> None:
+        """adama_debug_wgrad_expire_wait (test hook: a device-side wait that runs out and a
+        kernel that returns all the same).  Dense 2-D tensors as for linear_wgrad_fold."""
+        tokens, d_in = X.shape
+        d_out = dY.shape[1]
+        self._check(self._L.adama_debug_wgrad_expire_wait(
+            self._h, _dev_ptr(X, torch.bfloat16, "X"), _dev_ptr(dY, torch.bfloat16, "dY"),
+            tokens, d_in, d_out, X.stride(0), dY.stride(0), _dev_ptr(m, torch.float32, "m"),
+            _dev_ptr(v, torch.float32, "v"), m.stride(0), int(wait_limit_ns),
+            _stream_ptr(self.device)))
+
+    def debug_set_wgrad_variant(self, epilogue: int = 0, epi_warps: int = 0, box_loads: int = 0,
+                                no_pdl: int = 0, tile_cols: int = 0) -> None:
+        """adama_debug_set_wgrad_variant (test hook: pins the fused kernel's instance)."""
+        self._check(self._L.adama_debug_set_wgrad_variant(self._h, epilogue, epi_warps, box_loads,
+                                                          no_pdl, tile_cols))
+
     @property
     def launch_count(self) -> int:
         return int(self._L.adama_launch_count(self._h))
@@ -520,6 +544,12 @@ def linear_wgrad_fold_noalloc(X: torch.Tensor, dY: torch.Tensor, m: torch.Tensor
         _stream_ptr(torch.device("cuda", dev)))
     if st != 0:
         raise AdamAError(st, err.value.decode())
+
+
+def debug_setup_state(device: int) -> int:
+    """adama_debug_setup_state: bit 0 = tensor-map encoder resolved, bit 1 = kernel attributes
+    set on `device` (no GPU needed)."""
+    return int(load_library().adama_debug_setup_state(int(device)))
 
 
 def version() -> str:

@@ -21,6 +21,7 @@ struct adama_ctx {
     cudaEvent_t ev_copied[2], ev_folded[2], ev_entry;
     int64_t launches;
     double weight_decay;  // decoupled (AdamW) decay; 0 = the paper's plain update
+    adama::WgradVariant variant;  // adama_debug_set_wgrad_variant; all 0 = automatic
     char err[256];
 };
 
@@ -242,7 +243,8 @@ adama_status adama_fold(adama_ctx *ctx, const void *grad, adama_dtype gdt, float
 
 static adama_status wgrad_impl(adama_ctx *ctx, const void *X, const void *dY, int tokens, int d_in,
                                int d_out, int64_t ldx, int64_t ldy, float *m, float *v,
-                               int64_t ldmv, float *bias_m, float *bias_v, void *cuda_stream) {
+                               int64_t ldmv, float *bias_m, float *bias_v, void *cuda_stream,
+                               unsigned long long wait_limit_ns = 0, int withhold_last_load = 0) {
     adama_status st = check_wgrad_args(ctx, X, dY, tokens, d_in, d_out, ldx, ldy, m, v, ldmv);
     if (st != ADAMA_OK) return st;
     if (tokens == 0) return ADAMA_OK;  // empty sum: G = 0, nothing to add
@@ -264,6 +266,9 @@ static adama_status wgrad_impl(adama_ctx *ctx, const void *X, const void *dY, in
     a.stream = static_cast<cudaStream_t>(cuda_stream);
     a.bias_m = bias_m;
     a.bias_v = bias_v;
+    a.variant = ctx->variant;
+    a.wait_limit_ns = wait_limit_ns;
+    a.withhold_last_load = withhold_last_load;
     const char *msg = "wgrad_fold";
     cudaError_t e = adama::launch_wgrad_fold(a, &msg);
     if (e != cudaSuccess) return cuda_fail(ctx, msg, e);
@@ -701,6 +706,35 @@ adama_status adama_debug_set_status(adama_ctx *ctx, unsigned code, unsigned wait
     if (e != cudaSuccess) return cuda_fail(ctx, "debug_set_status", e);
     return ADAMA_OK;
 }
+
+adama_status adama_debug_wgrad_expire_wait(adama_ctx *ctx, const void *X, const void *dY,
+                                           int tokens, int d_in, int d_out, int64_t ldx, int64_t ldy,
+                                           float *m, float *v, int64_t ldmv, uint64_t wait_limit_ns,
+                                           void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (wait_limit_ns < 1000 || wait_limit_ns > 1000000000ull || tokens == 0)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG,
+                    "debug_wgrad_expire_wait: limit must be 1 us .. 1 s and tokens > 0");
+    return wgrad_impl(ctx, X, dY, tokens, d_in, d_out, ldx, ldy, m, v, ldmv, nullptr, nullptr,
+                      cuda_stream, wait_limit_ns, 1);
+}
+
+adama_status adama_debug_set_wgrad_variant(adama_ctx *ctx, int epilogue, int epi_warps,
+                                           int box_loads, int no_pdl, int tile_cols) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (epilogue < 0 || epilogue > 2 || (epi_warps != 0 && epi_warps != 4 && epi_warps != 8) ||
+        (box_loads != 0 && box_loads != 1) || (no_pdl != 0 && no_pdl != 1) || tile_cols < 0 ||
+        tile_cols > 256 || tile_cols % 32)
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "debug_set_wgrad_variant: value out of range");
+    ctx->variant.epilogue = epilogue;
+    ctx->variant.epi_warps = epi_warps;
+    ctx->variant.box_loads = box_loads;
+    ctx->variant.no_pdl = no_pdl;
+    ctx->variant.tile_cols = tile_cols;
+    return ADAMA_OK;
+}
+
+int adama_debug_setup_state(int device) { return adama::wgrad_setup_state(device); }
 
 const char *adama_last_error(const adama_ctx *ctx) { return ctx ? ctx->err : ""; }
 

@@ -90,6 +90,17 @@ cudaError_t launch_bias_grad_fold(const void *dY, int tokens, int d_out, int64_t
                                   float *v, FoldConstants c, cudaStream_t stream);
 
 // fused weight-gradient + fold (wgrad_fold.cu)
+// Which instance of the kernel a launch uses; 0 everywhere = chosen per launch from the shape.
+// Set through adama_debug_set_wgrad_variant so that the tests reach every instance on every
+// shape, whichever the automatic choice would be.
+struct WgradVariant {
+    int epilogue = 0;   // 1 = direct (accumulator -> registers -> m, v), 2 = staged through shared memory
+    int epi_warps = 0;  // 4 or 8 epilogue warps (direct epilogue)
+    int box_loads = 0;  // 1 = one TMA operation per 64-feature box even where grouped loads apply
+    int no_pdl = 0;     // 1 = plain stream order instead of programmatic dependent launch
+    int tile_cols = 0;  // width of the column tiles (multiple of 32, <= 256)
+};
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;  // 2 s per device-side wait
 struct WgradArgs {
     const void *X;
     const void *dY;
@@ -105,10 +116,16 @@ struct WgradArgs {
     // folded into them by the same launch
     float *bias_m = nullptr;
     float *bias_v = nullptr;
+    WgradVariant variant;
+    unsigned long long wait_limit_ns = 0;  // 0 = kDefaultWaitLimitNs
+    int withhold_last_load = 0;            // expiry test only: see adama_debug_wgrad_expire_wait
 };
 // Returns cudaSuccess or the failing CUDA error; *msg (static string) says which step failed.
 cudaError_t launch_wgrad_fold(const WgradArgs &args, const char **msg);
 // One-time, per process: resolves the driver's tensor-map encoder.
 cudaError_t wgrad_fold_setup(const char **msg);
+// Set-up bookkeeping, for diagnostics: bit 0 = the encoder has been resolved, bit 1 = the
+// kernels' attributes have been set on `device`.
+int wgrad_setup_state(int device);
 
 }  // namespace adama

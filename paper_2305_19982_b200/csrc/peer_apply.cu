@@ -1,7 +1,8 @@
 // State-sharded update with the exchange fused in: reduce-scatter of m and v, the update of
 // the owner's shard of w, and the all-gather of w, as ONE kernel over peer-mapped buffers
 // (NVLink / NVSwitch peer access: plain 128-bit loads and stores, no multicast, no waiting
-// inside the kernel).  Rank r's launch touches only shard r of every rank's w, m and v:
+// inside the kernel; the loads of up to 8 peers are issued together so that their round trips
+// overlap).  Rank r's launch touches only shard r of every rank's w, m and v:
 //   S_m = sum_q m_q[shard r],  S_v = sum_q v_q[shard r]            (rank order: deterministic)
 //   w_new = update(w_r, S_m / R, S_v / R^2)                        (Algorithm 2 "Update" on the
 //                                                                   averaged states, Eqs. 6-7)
@@ -16,6 +17,7 @@ namespace adama {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kPeerBatch = 8;  // peers whose m, v loads are in flight together (64 data registers)
 
 struct PeerTable {
     float *w[kMaxPeers];
@@ -44,13 +46,26 @@ apply_sharded_peers_kernel(const __grid_constant__ PeerTable tab, size_t lo4, si
     for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n4;
          i += (size_t)gridDim.x * kThreads) {
         const size_t e = (lo4 + i) * 4;
+        // All loads of a batch of peers are issued before the first add, so that their NVLink
+        // round trips overlap; the adds then run in rank order (deterministic, and the same
+        // sums as a serial loop over the peers).
         float4 sm = zero, sv = zero;
-        for (int q = 0; q < tab.world; ++q) {
-            const float4 a = ld4(tab.m[q] + e), b = ld4(tab.v[q] + e);
-            sm.x += a.x; sm.y += a.y; sm.z += a.z; sm.w += a.w;
-            sv.x += b.x; sv.y += b.y; sv.z += b.z; sv.w += b.w;
-        }
         float4 w = ld4(tab.w[tab.rank] + e);
+        for (int q0 = 0; q0 < tab.world; q0 += kPeerBatch) {
+            float4 a[kPeerBatch], b[kPeerBatch];
+#pragma unroll
+            for (int j = 0; j < kPeerBatch; ++j)
+                if (q0 + j < tab.world) {
+                    a[j] = ld4(tab.m[q0 + j] + e);
+                    b[j] = ld4(tab.v[q0 + j] + e);
+                }
+#pragma unroll
+            for (int j = 0; j < kPeerBatch; ++j)
+                if (q0 + j < tab.world) {
+                    sm.x += a[j].x; sm.y += a[j].y; sm.z += a[j].z; sm.w += a[j].w;
+                    sv.x += b[j].x; sv.y += b[j].y; sv.z += b[j].z; sv.w += b[j].w;
+                }
+        }
         apply1(w.x, sm.x, sv.x, c);
         apply1(w.y, sm.y, sv.y, c);
         apply1(w.z, sm.z, sv.z, c);

@@ -47,7 +47,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include <cstdlib>
+#include <mutex>
 
 #include "adama_internal.h"
 
@@ -102,8 +102,10 @@ constexpr int STAGED_STREAM_WARPS = 8;  // shared memory -> m, v (16 rows of the
 constexpr int G_TILE_BYTES = 2 * PART_BYTES;  // two parts: one is filled while the other is folded
 constexpr int STAGED_THREADS = 32 * (2 + STAGED_DRAIN_WARPS + STAGED_STREAM_WARPS + BIAS_WARPS);
 
-// Per-variant geometry: CTAS = CTAs cooperating on one tile (1 or 2).
-template <int CTAS, bool STAGED = false>
+constexpr int CTAS = 2;  // CTAs cooperating on one tile (tcgen05 cta_group::2)
+
+// Per-variant geometry (STAGED: the short-call instance with the staged epilogue).
+template <bool STAGED = false>
 struct Geo {
     static constexpr int ROWS_PER_CTA = 128;                 // TMEM lanes
     static constexpr int TILE_M = ROWS_PER_CTA * CTAS;       // UMMA M
@@ -114,7 +116,7 @@ struct Geo {
     static constexpr int B_STAGE_BYTES = B_BOXES * BOX_BYTES;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KB or 32 KB
     static constexpr int STAGES =
-        STAGED ? STAGED_RING : (CTAS == 1 ? 4 * 64 / BK : ADAMA_WGRAD_STAGES);
+        STAGED ? STAGED_RING : ADAMA_WGRAD_STAGES;
     static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + (STAGED ? G_TILE_BYTES : EPI_BYTES);
     static constexpr int SMEM_BIAS_OFF = SMEM_BAR_OFF + SMEM_BAR_BYTES;
@@ -132,7 +134,6 @@ struct Geo {
                                                 | ((uint32_t)(TILE_M >> 4) << 24);
 };
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr unsigned long long kDrainLimitNs = 20000000ull;   // 20 ms
 
 // ---- PTX wrappers --------------------------------------------------------------------------
@@ -187,7 +188,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: false if `limit_ns` passed or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          unsigned long long limit_ns = kWaitLimitNs) {
+                                          unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer();
     for (uint32_t spins = 1;; ++spins) {
@@ -198,43 +199,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
-// TMA tile load into this CTA's shared memory; `bar` is a shared::cluster address and,
-// for CTAS == 2, may name the partner CTA's barrier.
-template <int CTAS>
+// TMA tile load into this CTA's shared memory; `bar` is a shared::cluster address and may
+// name the partner CTA's barrier.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
                                             uint32_t bar) {
-    if constexpr (CTAS == 1) {
-        asm volatile(
-            "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-            "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-            "l"(map), "r"(x), "r"(y), "r"(bar)
-            : "memory");
-    } else {
-        asm volatile(
-            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-            "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-            "l"(map), "r"(x), "r"(y), "r"(bar)
-            : "memory");
-    }
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
 }
 // Same, through a 3-D view {64 features, tokens, 64-feature groups}: one operation brings
 // several 64-feature groups (boxes of 8192 bytes, one after the other in shared memory).
-template <int CTAS>
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int tok, int grp,
                                             uint32_t bar) {
-    if constexpr (CTAS == 1) {
-        asm volatile(
-            "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-            "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-            "l"(map), "r"(0), "r"(tok), "r"(grp), "r"(bar)
-            : "memory");
-    } else {
-        asm volatile(
-            "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-            "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-            "l"(map), "r"(0), "r"(tok), "r"(grp), "r"(bar)
-            : "memory");
-    }
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(0), "r"(tok), "r"(grp), "r"(bar)
+        : "memory");
 }
 // Programmatic dependent launch.  grid_dependency_wait: returns once the kernel launched before
 // this one in the stream has completed and its writes are visible (at once if this launch was
@@ -258,60 +241,29 @@ __device__ __forceinline__ void tc_fence_after() {
 }
 // Arrive on `cluster_bar` (shared::cluster address) once all MMAs issued so far by this
 // thread have retired.
-template <int CTAS>
 __device__ __forceinline__ void tc_commit(uint32_t cluster_bar) {
-    if constexpr (CTAS == 1) {
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                         cluster_bar)
-                     : "memory");
-    } else {
-        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                         cluster_bar)
-                     : "memory");
-    }
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                     cluster_bar)
+                 : "memory");
 }
-template <int CTAS>
 __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b,
                                        uint32_t idesc, uint32_t accumulate) {
-    if constexpr (CTAS == 1) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-            "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-            "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-            : "memory");
-    }
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
-template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem) {
-    if constexpr (CTAS == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
-                     "n"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    } else {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
-                     "n"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                 "n"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
-template <int CTAS>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr) {
-    if constexpr (CTAS == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "n"(TMEM_COLS)
-                     : "memory");
-    } else {
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "n"(TMEM_COLS)
-                     : "memory");
-    }
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "n"(TMEM_COLS)
+                 : "memory");
 }
 // 32 lanes x 32 consecutive fp32 columns: thread i receives TMEM lane (base lane + i).
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -394,9 +346,13 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= SMEM_BAR_BYTES, "barrier block");
 
+// The status block is global memory that the previous kernel of the stream (or the host's
+// clearing of it) may still be writing under programmatic launch: the report waits for that
+// kernel first (a no-op for roles that already have).
 __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars, unsigned site,
                                                unsigned tile) {
     *reinterpret_cast<volatile int *>(&bars->abort_flag) = 1;
+    grid_dependency_wait();
     if (atomicCAS(status, (unsigned)kDevOk, (unsigned)kDevTimeout) == kDevOk) {
         status[1] = site;
         status[2] = tile;
@@ -415,7 +371,6 @@ __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars,
 struct WorkItem {
     int m0, n0, width;
 };
-template <int CTAS>
 __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m, int tiles_n) {
     int full = w, half = 0, width = BN;
     if (w >= split_from) {
@@ -426,10 +381,10 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
     }
     const int tm = tiles_n < tiles_m ? full / tiles_n : full % tiles_m;
     const int tn = tiles_n < tiles_m ? full % tiles_n : full / tiles_m;
-    return {tm * Geo<CTAS>::TILE_M, tn * BN + half * (BN / 2), width};
+    return {tm * Geo<>::TILE_M, tn * BN + half * (BN / 2), width};
 }
 
-template <int CTAS, bool STAGED>
+template <bool STAGED>
 __global__ void __launch_bounds__(STAGED ? STAGED_THREADS : MAX_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   const __grid_constant__ CUtensorMap map_dy,
@@ -440,8 +395,9 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                   float *__restrict__ v_out, long long ldmv, int tokens, int d_in, int d_out,
                   int split_from, int num_items, float a, float b, unsigned *status,
                   const __nv_bfloat16 *__restrict__ dy_raw, long long ldy,
-                  float *__restrict__ bias_m, float *__restrict__ bias_v) {
-    using G = Geo<CTAS, STAGED>;
+                  float *__restrict__ bias_m, float *__restrict__ bias_v,
+                  unsigned long long wait_limit_ns, int withhold_last_load) {
+    using G = Geo<STAGED>;
     constexpr int STAGES = G::STAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -452,7 +408,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t rank = (CTAS == 1) ? 0u : cluster_ctarank();  // position in the pair
+    const uint32_t rank = cluster_ctarank();  // position in the pair
     const int group = blockIdx.x / CTAS;                           // which pair
     const int num_groups = gridDim.x / CTAS;
     const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
@@ -482,10 +438,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
     }
-    if (warp == 1) tmem_alloc<CTAS>(smem_u32(&bars->tmem_base));
+    if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base));
     tc_fence_before();
     __syncthreads();
-    if constexpr (CTAS == 2) cluster_sync_all();  // the partner's barriers exist before anyone signals them
+    cluster_sync_all();  // the partner's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
     // Everything above touched only this CTA's shared and tensor memory, so it may run while
@@ -505,9 +461,9 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             bool ok = true;
             const uint32_t full0 = smem_u32(&bars->full[0]);
             // the pair's loads are counted by the first CTA's barrier
-            const uint32_t full0_lead = (CTAS == 1) ? full0 : map_to_cta(full0, 0);
+            const uint32_t full0_lead = map_to_cta(full0, 0);
             for (int tile = group; tile < num_items && ok; tile += num_groups) {
-                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
+                const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
                 const int cols_per_cta = wi.width / CTAS;  // dY columns this CTA stages
                 const int b_boxes = cols_per_cta / GROUP;
                 const int m0 = wi.m0 + (int)rank * G::ROWS_PER_CTA;
@@ -515,11 +471,14 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 const uint32_t stage_tx =
                     (uint32_t)(G::A_STAGE_BYTES + b_boxes * BOX_BYTES) * CTAS;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
+                    ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag, wait_limit_ns);
                     if (!ok) {
                         record_timeout(status, bars, 1, (unsigned)tile);
                         break;
                     }
+                    // Test hook (adama_debug_wgrad_expire_wait): the last stage of the launch's
+                    // last work item is never loaded, so the issuer's wait for it must run out.
+                    if (withhold_last_load && kb == num_kb - 1 && tile == num_items - 1) break;
                     const uint32_t bar = full0_lead + (uint32_t)stage * 8u;
                     const uint32_t sa = base + stage * G::STAGE_BYTES;
                     const uint32_t sb = sa + G::A_STAGE_BYTES;
@@ -527,16 +486,16 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     if (rank == 0) mbar_arrive_expect_tx(full0 + (uint32_t)stage * 8u, stage_tx);
                     if (grouped) {
                         // d_in, d_out multiples of 64: one operation per operand
-                        tma_load_3d<CTAS>(sa, &map_x3, kb * BK, m0 / GROUP, bar);
-                        tma_load_3d<CTAS>(sb, b_boxes == G::B_BOXES ? &map_dy3 : &map_dy3h, kb * BK,
+                        tma_load_3d(sa, &map_x3, kb * BK, m0 / GROUP, bar);
+                        tma_load_3d(sb, b_boxes == G::B_BOXES ? &map_dy3 : &map_dy3h, kb * BK,
                                           n0 / GROUP, bar);
                     } else {
 #pragma unroll
                         for (int j = 0; j < G::A_BOXES; ++j)
-                            tma_load_2d<CTAS>(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK,
+                            tma_load_2d(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK,
                                               bar);
                         for (int j = 0; j < b_boxes; ++j)
-                            tma_load_2d<CTAS>(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK,
+                            tma_load_2d(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK,
                                               bar);
                     }
                     armed |= 1u << stage;
@@ -572,16 +531,15 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             uint32_t empty_bar0[CTAS];  // empty[0] in each CTA of the pair
 #pragma unroll
             for (int r = 0; r < CTAS; ++r)
-                empty_bar0[r] = CTAS == 1 ? smem_u32(&bars->empty[0])
-                                          : map_to_cta(smem_u32(&bars->empty[0]), r);
+                empty_bar0[r] = map_to_cta(smem_u32(&bars->empty[0]), r);
             bool next_ready = false;  // full[stage] already seen complete by a probe
             for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
                 const uint32_t idesc =
                     G::INSTR_DESC_NO_N |
-                    ((uint32_t)(work_item<CTAS>(tile, split_from, tiles_m, tiles_n).width >> 3) << 17);
-                ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag);
+                    ((uint32_t)(work_item(tile, split_from, tiles_m, tiles_n).width >> 3) << 17);
+                ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag, wait_limit_ns);
                 if (!ok) {
                     record_timeout(status, bars, 2, (unsigned)tile);
                     break;
@@ -590,7 +548,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!next_ready) {
-                        ok = mbar_wait(full0 + (uint32_t)stage * 8u, phase, abort_flag);
+                        ok = mbar_wait(full0 + (uint32_t)stage * 8u, phase, abort_flag, wait_limit_ns);
                         if (!ok) {
                             record_timeout(status, bars, 3, (unsigned)tile);
                             break;
@@ -610,29 +568,29 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     constexpr int KSTEPS = BK / UMMA_K;
 #pragma unroll
                     for (int k = 0; k < KSTEPS - 1; ++k)
-                        tc_mma<CTAS>(tmem_d, smem_desc(a_lo + k * kstep),
+                        tc_mma(tmem_d, smem_desc(a_lo + k * kstep),
                                      smem_desc(b_lo + k * kstep), idesc, (kb | k) != 0 ? 1u : 0u);
                     // look ahead while those execute (a stale "ready" cannot occur: the
                     // barrier cannot advance two phases before this thread frees the stage)
                     next_ready = mbar_try_wait(full0 + (uint32_t)nstage * 8u, nphase);
-                    tc_mma<CTAS>(tmem_d, smem_desc(a_lo + (KSTEPS - 1) * kstep),
+                    tc_mma(tmem_d, smem_desc(a_lo + (KSTEPS - 1) * kstep),
                                  smem_desc(b_lo + (KSTEPS - 1) * kstep), idesc, 1u);
                     // the stage is free, in every CTA of the pair, once these MMAs retire
 #pragma unroll
                     for (int r = 0; r < CTAS; ++r)
-                        tc_commit<CTAS>(empty_bar0[r] + (uint32_t)stage * 8u);
+                        tc_commit(empty_bar0[r] + (uint32_t)stage * 8u);
                     stage = nstage;
                     phase = nphase;
                 }
                 if (ok) {
                     const uint32_t f = smem_u32(&bars->acc_full[as]);
 #pragma unroll
-                    for (int r = 0; r < CTAS; ++r) tc_commit<CTAS>(CTAS == 1 ? f : map_to_cta(f, r));
+                    for (int r = 0; r < CTAS; ++r) tc_commit(map_to_cta(f, r));
                 }
             }
             if (*abort_flag) {
                 // let issued MMAs retire before TMEM is given back
-                tc_commit<CTAS>(smem_u32(&bars->drain));
+                tc_commit(smem_u32(&bars->drain));
                 int never = 0;
                 mbar_wait(smem_u32(&bars->drain), 0, &never, kDrainLimitNs);
             }
@@ -654,12 +612,12 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         uint32_t use_bits = 0;    // bit k: parity of how often part buffer k has been used
         grid_dependency_wait();   // m and v may still be written by the previous call
         for (int tile = group; tile < num_items && ok; tile += num_groups) {
-            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
+            const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
             const int row_base = wi.m0 + (int)rank * G::ROWS_PER_CTA;
             for (int part_i = 0; part_i < wi.width / PART_COLS; ++part_i) {
                 if (!ok) continue;
                 const int k = part_i & 1;
-                ok = mbar_wait(smem_u32(&bars->g_full[k]), (use_bits >> k) & 1u, abort_flag);
+                ok = mbar_wait(smem_u32(&bars->g_full[k]), (use_bits >> k) & 1u, abort_flag, wait_limit_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) {
                     if (lane == 0) record_timeout(status, bars, 7, (unsigned)tile);
@@ -815,8 +773,8 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-                const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
-                ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
+                const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
+                ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag, wait_limit_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) {
                     if (lane == 0) record_timeout(status, bars, 4, (unsigned)tile);
@@ -829,7 +787,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     if (!ok) continue;
                     const int k = part_i & 1;
                     // the streaming warps must be done with this buffer's previous contents
-                    ok = mbar_wait(smem_u32(&bars->g_empty[k]), ((use_bits >> k) & 1u) ^ 1u, abort_flag);
+                    ok = mbar_wait(smem_u32(&bars->g_empty[k]), ((use_bits >> k) & 1u) ^ 1u, abort_flag, wait_limit_ns);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) {
                         if (lane == 0) record_timeout(status, bars, 6, (unsigned)tile);
@@ -858,8 +816,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 __syncwarp();
                 if (lane == 0) {
                     const uint32_t e = smem_u32(&bars->acc_empty[as]);
-                    if constexpr (CTAS == 1) mbar_arrive(e);
-                    else mbar_arrive_cluster(map_to_cta(e, 0));
+                    mbar_arrive_cluster(map_to_cta(e, 0));
                 }
             }
         } else {
@@ -881,10 +838,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-            const WorkItem wi = work_item<CTAS>(tile, split_from, tiles_m, tiles_n);
+            const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
             const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
             const int chunks = wi.width / (col_split * EPI_COLS);  // chunks per warp
-            ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag);
+            ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag, wait_limit_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
                 if (lane == 0) record_timeout(status, bars, 4, (unsigned)tile);
@@ -959,8 +916,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             __syncwarp();
             if (lane == 0) {
                 const uint32_t e = smem_u32(&bars->acc_empty[as]);
-                if constexpr (CTAS == 1) mbar_arrive(e);
-                else mbar_arrive_cluster(map_to_cta(e, 0));
+                mbar_arrive_cluster(map_to_cta(e, 0));
             }
         }
         }  // !STAGED
@@ -970,10 +926,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     __syncthreads();
     // neither CTA of a pair may retire while the other can still read its shared memory
     // or signal its barriers
-    if constexpr (CTAS == 2) cluster_sync_all();
+    cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc<CTAS>(tmem_base);
+        tmem_dealloc(tmem_base);
     }
 }
 
@@ -984,12 +940,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
-bool g_attr_set = false;
-int g_variant = 0;  // 0 = not chosen yet, 1 = one-CTA tiles, 2 = CTA pairs
-bool g_no_grouped = false;
-int g_force_epi_warps = 0;  // ADAMA_WGRAD_EPI_WARPS=4|8 overrides the per-launch choice (comparisons)
-bool g_no_pdl = false;
-int g_force_staged = 0;  // ADAMA_WGRAD_STAGED=1|0 forces / forbids the staged epilogue (comparisons)
+// One-time set-up, guarded by g_setup_mutex: the driver's tensor-map encoder once per process,
+// the kernels' shared-memory limit once per DEVICE (cudaFuncSetAttribute applies to the
+// current device only).
+std::mutex g_setup_mutex;
+constexpr int kMaxTrackedDevices = 64;
+bool g_attr_set[kMaxTrackedDevices] = {};
 
 // 2-D row-major tensor [rows, cols] with row pitch `ld` elements, box [box_rows, box_cols].
 bool encode_2d(CUtensorMap *map, CUtensorMapDataType dt, size_t elem, const void *ptr,
@@ -1024,6 +980,7 @@ bool encode_grouped(CUtensorMap *map, const void *ptr, uint64_t d, uint64_t toke
 }  // namespace
 
 cudaError_t wgrad_fold_setup(const char **msg) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_encode) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -1039,42 +996,46 @@ cudaError_t wgrad_fold_setup(const char **msg) {
         }
         g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    if (!g_variant) {
-        // ADAMA_WGRAD_CTAS=1 selects the one-CTA tiling (for comparisons); default: pairs
-        const char *env = getenv("ADAMA_WGRAD_CTAS");
-        g_variant = (env && env[0] == '1') ? 1 : 2;
-        const char *ng = getenv("ADAMA_WGRAD_NO_GROUPED");
-        g_no_grouped = ng && ng[0] == '1';
-        const char *ew = getenv("ADAMA_WGRAD_EPI_WARPS");
-        g_force_epi_warps = ew && (ew[0] == '4' || ew[0] == '8') ? ew[0] - '0' : 0;
-        // ADAMA_WGRAD_NO_PDL=1 launches without programmatic stream serialization (comparisons)
-        const char *np = getenv("ADAMA_WGRAD_NO_PDL");
-        g_no_pdl = np && np[0] == '1';
-        const char *sg = getenv("ADAMA_WGRAD_STAGED");
-        g_force_staged = sg ? (sg[0] == '1' ? 1 : -1) : 0;
+    return cudaSuccess;
+}
+
+static bool attr_needed(int device) {
+    return device < 0 || device >= kMaxTrackedDevices || !g_attr_set[device];
+}
+
+int wgrad_setup_state(int device) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    return (g_encode ? 1 : 0) | (attr_needed(device) ? 0 : 2);
+}
+
+// The kernels' dynamic shared-memory limit on the CURRENT device (set once per device).
+static cudaError_t ensure_device_attributes(const char **msg) {
+    int device = -1;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) {
+        *msg = "cudaGetDevice";
+        return e;
     }
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!attr_needed(device)) return cudaSuccess;
+    e = cudaFuncSetAttribute(wgrad_fold_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Geo<false>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(wgrad_fold_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Geo<true>::SMEM_BYTES);
+    if (e != cudaSuccess) {
+        *msg = "cudaFuncSetAttribute(wgrad_fold_kernel)";
+        return e;
+    }
+    // devices beyond the table are simply set up on every call
+    if (device >= 0 && device < kMaxTrackedDevices) g_attr_set[device] = true;
     return cudaSuccess;
 }
 
 cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cudaError_t e = wgrad_fold_setup(msg);
+    if (e == cudaSuccess) e = ensure_device_attributes(msg);
     if (e != cudaSuccess) return e;
-    if (!g_attr_set) {
-        e = cudaFuncSetAttribute(wgrad_fold_kernel<1, false>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<1>::SMEM_BYTES);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(wgrad_fold_kernel<2, false>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::SMEM_BYTES);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(wgrad_fold_kernel<2, true>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     Geo<2, true>::SMEM_BYTES);
-        if (e != cudaSuccess) {
-            *msg = "cudaFuncSetAttribute(wgrad_fold_kernel)";
-            return e;
-        }
-        g_attr_set = true;
-    }
     CUtensorMap map_x, map_dy;
     bool ok = encode_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.X, (uint64_t)p.d_in,
                         (uint64_t)p.tokens, (uint64_t)p.ldx, GROUP, BK,
@@ -1082,25 +1043,24 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
               encode_2d(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.dY, (uint64_t)p.d_out,
                         (uint64_t)p.tokens, (uint64_t)p.ldy, GROUP, BK,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
-    // grouped loads need whole 64-feature groups in both operands (CTA-pair kernel only)
+    // grouped loads need whole 64-feature groups in both operands
     CUtensorMap map_x3 = map_x, map_dy3 = map_dy, map_dy3h = map_dy;
-    int grouped = (g_variant == 2 && p.d_in % GROUP == 0 && p.d_out % GROUP == 0 && !g_no_grouped) ? 1 : 0;
+    int grouped = (p.d_in % GROUP == 0 && p.d_out % GROUP == 0 && !p.variant.box_loads) ? 1 : 0;
     if (ok && grouped)
         ok = encode_grouped(&map_x3, p.X, (uint64_t)p.d_in, (uint64_t)p.tokens, (uint64_t)p.ldx, BK,
-                            Geo<2>::A_BOXES) &&
+                            Geo<>::A_BOXES) &&
              encode_grouped(&map_dy3, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens, (uint64_t)p.ldy,
-                            BK, Geo<2>::B_BOXES) &&
+                            BK, Geo<>::B_BOXES) &&
              encode_grouped(&map_dy3h, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens,
-                            (uint64_t)p.ldy, BK, Geo<2>::B_BOXES / 2);
+                            (uint64_t)p.ldy, BK, Geo<>::B_BOXES / 2);
     if (!ok) {
         *msg = "cuTensorMapEncodeTiled rejected a tensor";
         return cudaErrorInvalidValue;
     }
     const int tiles_n = (p.d_out + BN - 1) / BN;
     *msg = "wgrad_fold launch";
-    const int tile_m = g_variant == 1 ? Geo<1>::TILE_M : Geo<2>::TILE_M;
-    const int tiles = ((p.d_in + tile_m - 1) / tile_m) * tiles_n;
-    const int max_groups = g_variant == 1 ? p.sm_count : p.sm_count / 2;
+    const int tiles = ((p.d_in + Geo<>::TILE_M - 1) / Geo<>::TILE_M) * tiles_n;
+    const int max_groups = p.sm_count / 2;
     // Tail balancing: if the last round would keep at most half of the groups busy, its
     // tiles are issued as 128-column halves (see WorkItem).
     const int rest = tiles % max_groups;
@@ -1113,16 +1073,9 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     // 8 epilogue warps when no CTA group gets a second tile (exposed epilogue) or when the
     // contraction is short (up to 2048 tokens the m, v traffic of the epilogue, not the tensor
     // cores, bounds the call: 4096x4096 with 1024 tokens 78.9 vs 82.9 us), else 4
-    const bool wide = g_force_epi_warps ? g_force_epi_warps == 8
-                                        : (items <= max_groups || p.tokens <= 2048);
+    const bool wide = p.variant.epi_warps ? p.variant.epi_warps == 8
+                                          : (items <= max_groups || p.tokens <= 2048);
     const int threads = 32 * (2 + (wide ? MAX_EPI_WARPS : 4) + (p.bias_m ? BIAS_WARPS : 0));
-    if (g_variant == 1) {
-        wgrad_fold_kernel<1, false><<<groups, threads, Geo<1>::SMEM_BYTES, p.stream>>>(
-            map_x, map_dy, map_x3, map_dy3, map_dy3h, 0, p.m, p.v, (long long)p.ldmv, p.tokens,
-            p.d_in, p.d_out, split_from, items, p.c.a, p.c.b, p.status,
-            static_cast<const __nv_bfloat16 *>(p.dY), (long long)p.ldy, p.bias_m, p.bias_v);
-        return cudaGetLastError();
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
@@ -1130,8 +1083,8 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     // (4096x4096, L2 flushed, staged vs direct epilogue, us: 256 tokens 65.6 vs 75.8, 1024: 69.7 vs
     // 79.9, 2048: 75.8 vs 82.0, 3072: 94.2 vs 92.2, 4096: 114.7 vs 110.6.  With 128-column parts and
     // the 3-stage ring they leave: 66.6, 71.7, 92.2 at 256, 1024, 2048 tokens.)
-    const bool staged = g_force_staged ? g_force_staged > 0 : p.tokens <= 2048;
-    cfg.dynamicSmemBytes = staged ? Geo<2, true>::SMEM_BYTES : Geo<2>::SMEM_BYTES;
+    const bool staged = p.variant.epilogue ? p.variant.epilogue == 2 : p.tokens <= 2048;
+    cfg.dynamicSmemBytes = staged ? Geo<true>::SMEM_BYTES : Geo<>::SMEM_BYTES;
     if (staged) cfg.blockDim = dim3((unsigned)(STAGED_THREADS - (p.bias_m ? 0 : 32 * BIAS_WARPS)), 1, 1);
     cfg.stream = p.stream;
     cudaLaunchAttribute attr[2];
@@ -1143,12 +1096,13 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_no_pdl ? 1 : 2;
-    return cudaLaunchKernelEx(&cfg, staged ? wgrad_fold_kernel<2, true> : wgrad_fold_kernel<2, false>, map_x, map_dy, map_x3, map_dy3, map_dy3h,
-                              grouped, p.m, p.v,
+    cfg.numAttrs = p.variant.no_pdl ? 1 : 2;
+    const unsigned long long limit = p.wait_limit_ns ? p.wait_limit_ns : kDefaultWaitLimitNs;
+    return cudaLaunchKernelEx(&cfg, staged ? wgrad_fold_kernel<true> : wgrad_fold_kernel<false>,
+                              map_x, map_dy, map_x3, map_dy3, map_dy3h, grouped, p.m, p.v,
                               (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
                               p.c.a, p.c.b, p.status, static_cast<const __nv_bfloat16 *>(p.dY),
-                              (long long)p.ldy, p.bias_m, p.bias_v);
+                              (long long)p.ldy, p.bias_m, p.bias_v, limit, p.withhold_last_load);
 }
 
 }  // namespace adama
@@ -1176,10 +1130,12 @@ struct StaticSetup {
     int sm_count = 0;
 };
 StaticSetup g_static_setup[kMaxDevices];
+std::mutex g_static_mutex;  // the table is filled in by whichever thread calls first
 
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel
 // can use; the device address has to be asked for, with the right device current.
 cudaError_t static_setup_for_current_device(int device, StaticSetup **out, const char **msg) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
     StaticSetup &s = g_static_setup[device];
     if (!s.scratch) {
         void *ptr = nullptr;

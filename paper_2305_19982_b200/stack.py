@@ -62,38 +62,34 @@ class LinearStack:
     def flops_per_micro_batch(self, tokens: int) -> float:
         return sum(2.0 * tokens * L.d_in * L.d_out for L in self.layers)
 
-    def minibatch(self, opt: AdamA, n_micro: int, lr: float,
-                  inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]],
-                  materialise: str = "none") -> None:
-        """One mini-batch.  `inputs(micro, layer_index, spec)` returns (X, dY) for that
-        (micro-batch, layer); the tensors are released right after the layer's call.
-
-        materialise: "none"  -- fused kernel, the weight gradient never exists in memory;
-                     "layer" -- the paper's pipeline: a per-layer fp32 gradient buffer is
-                                assigned, filled by a library GEMM, folded with adama_fold
-                                and released (for memory / speed comparison only).
-        """
+    def fold_micro_batches(self, opt: AdamA, n_micro: int,
+                           inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]]) -> None:
+        """The accumulation half of one mini-batch (Algorithm 2, inner loops): begin, then for
+        every micro-batch every layer from the last to the first through the fused
+        weight-gradient fold.  `inputs(micro, layer_index, spec)` returns (X, dY) for that
+        (micro-batch, layer); the tensors are released right after the layer's call.  The
+        weight gradient never exists in memory.  On return m, v hold m_t, v_t."""
         opt.begin_minibatch(n_micro)
         for i in range(n_micro):
             for j in reversed(range(len(self.layers))):
-                spec = self.layers[j]
-                X, dY = inputs(i, j, spec)
-                if materialise == "none":
-                    if self.biases:  # bias gradient (column sums of dY) in the same launch
-                        opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j),
-                                              self.bias_view(self.m, j), self.bias_view(self.v, j))
-                    else:
-                        opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j))
+                X, dY = inputs(i, j, self.layers[j])
+                if self.biases:  # bias gradient (column sums of dY) in the same launch
+                    opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j),
+                                          self.bias_view(self.m, j), self.bias_view(self.v, j))
                 else:
-                    G = torch.empty(spec.d_in, spec.d_out, dtype=torch.float32, device=self.device)
-                    torch.mm(X.t(), dY, out_dtype=torch.float32, out=G)
-                    opt.fold(G.view(-1), self.view(self.m, j).view(-1), self.view(self.v, j).view(-1))
-                    del G
-                    if self.biases:
-                        opt.bias_grad_fold(dY, self.bias_view(self.m, j), self.bias_view(self.v, j))
+                    opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j))
                 del X, dY
-        # one apply over the whole flat buffer (padding between layers holds zeros)
+
+    def apply(self, opt: AdamA, lr: float) -> None:
+        """The update half (Algorithm 2, "Update"): one apply over the whole flat buffer (the
+        padding between layers holds zeros); m, v leave it decayed for the next mini-batch."""
         opt.apply(self.w, self.m, self.v, lr)
+
+    def minibatch(self, opt: AdamA, n_micro: int, lr: float,
+                  inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]]) -> None:
+        """One whole mini-batch: fold_micro_batches, then apply."""
+        self.fold_micro_batches(opt, n_micro, inputs)
+        self.apply(opt, lr)
 
 
 def gpt2xl_stack(blocks: int, device="cuda", biases: bool = False) -> LinearStack:

@@ -85,3 +85,14 @@ def test_init_without_gpu_fails_loudly():
         pytest.skip("a GPU is present")
     with pytest.raises(adama.AdamAError):
         adama.AdamA()
+
+
+def test_setup_bookkeeping_is_per_device_and_starts_empty():
+    """The fused kernel's attributes are per device: the table that remembers them answers
+    "not set up" for every device no launch has run on, and for ordinals outside the table
+    (those are set up on every call).  No GPU needed: nothing has been launched here."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("another test in this process may already have launched on device 0")
+    for dev in (0, 1, 7, 63, 64, 1000, -1):
+        assert adama.debug_setup_state(dev) & 2 == 0

@@ -19,20 +19,53 @@ def test_headline_step_byte_and_flop_counts():
     assert flops == 4 * 2.0 * 4096 ** 3
 
 
-def test_traffic_entry_is_dropped_when_a_source_changes(tmp_path, monkeypatch):
+def test_traffic_entry_is_scaled_to_the_run_and_dropped_when_a_source_changes(tmp_path, monkeypatch):
     src = tmp_path / "k.cu"
     src.write_text("kernel v1")
     prof = tmp_path / "profiles"
     prof.mkdir()
-    entry = {"bytes_per_launch": 123, "sources": ["k.cu"],
-             "sha256": hashlib.sha256(b"kernel v1").hexdigest()}
-    (prof / "traffic.json").write_text(json.dumps({"_note": "x", "fold_bf16": entry}))
+    sha = hashlib.sha256(b"kernel v1").hexdigest()
+    table = {"_note": "x",
+             "fold_bf16": {"captured_params": 1000, "captured_bytes": 17000, "sources": ["k.cu"], "sha256": sha},
+             "wgrad_fold": {"shape": [64, 128, 256], "captured_bytes": 555, "sources": ["k.cu"], "sha256": sha}}
+    (prof / "traffic.json").write_text(json.dumps(table))
     monkeypatch.setattr(bench, "ROOT", tmp_path)
-    assert bench.load_traffic() == {"fold_bf16": 123}
+    got = bench.load_traffic(5000, 64, 128, 256)
+    assert got["fold_bf16"]["bytes_per_launch"] == 85000      # scaled by this run's size
+    assert "lower bound" in got["fold_bf16"]["note"] and "1000-param" in got["fold_bf16"]["note"]
+    assert got["wgrad_fold"]["bytes_per_launch"] == 555
+    assert "wgrad_fold" not in bench.load_traffic(5000, 64, 128, 512)   # another shape: no figure
     src.write_text("kernel v2")
-    assert bench.load_traffic() == {}
+    assert bench.load_traffic(5000, 64, 128, 256) == {}
     (prof / "traffic.json").write_text("not json")
-    assert bench.load_traffic() == {}
+    assert bench.load_traffic(5000, 64, 128, 256) == {}
+
+
+def test_one_oracle_sample_serves_both_arms():
+    """The cpu_baseline of the default run and the --impl reference arm time the oracle on the
+    same bounded sample of the headline step."""
+    import inspect
+    src = inspect.getsource(bench)
+    assert src.count("time_oracle(*ORACLE_SAMPLE") == 2
+    assert bench.ORACLE_SAMPLE == (1 << 24, 256, 512, 512)
+
+
+def test_gpus_flag_without_a_launcher_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment re-launches itself as
+    two ranks (gloo here, no GPU work) and prints ONE line that says n_gpus: 2."""
+    import os
+    import subprocess
+    import sys
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, str(bench.ROOT / "bench.py"), "--gpus", "2",
+                          "--workload", "launch_check", "--backend", "gloo"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["metric"] == "launch_check"
+    assert line["ms_per_step"] >= 20.0      # the max over the ranks (rank 1 sleeps 20 ms)
 
 
 def test_peaks_come_from_the_measured_file_when_present(tmp_path, monkeypatch):

@@ -176,3 +176,70 @@ def test_bench_reference_arm_under_torchrun_prints_one_line():
     assert len(lines) == 1
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
+
+
+def _peer_states_rank(rank, world, port, out_dir):
+    """PeerMappedStates with stand-ins for torch's symmetric memory (CPU tensors, made-up peer
+    addresses) and for the optimizer: what is checked is the protocol around the one fused
+    launch -- padding rule, zeroed accumulators, barrier / launch / barrier order, this rank's
+    index and every rank's w, m, v addresses handed to adama_apply_sharded_peers."""
+    import types
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    log = []
+
+    class Handle:
+        def __init__(self, t, tag):
+            self.buffer_ptrs = [1000 * tag + q for q in range(world)]
+            self.tag = tag
+
+        def barrier(self):
+            dist.barrier()
+            log.append(("barrier", self.tag))
+
+    made = []
+
+    def empty(n, dtype, device):
+        t = torch.full((n,), 7.0, dtype=dtype)
+        made.append(t)
+        return t
+
+    fake = types.ModuleType("torch.distributed._symmetric_memory")
+    fake.empty = empty
+    fake.rendezvous = lambda t, group: Handle(t, len(made))
+    sys.modules["torch.distributed._symmetric_memory"] = fake
+    torch.distributed._symmetric_memory = fake
+
+    class Opt:
+        def apply_sharded_peers(self, w_ptrs, m_ptrs, v_ptrs, r, n, lr):
+            log.append(("launch", list(w_ptrs), list(m_ptrs), list(v_ptrs), r, n, lr))
+
+    ok = True
+    try:
+        ddp.PeerMappedStates(4 * world + 4, "cpu")     # not a multiple of 4 * world
+        ok = False
+    except ValueError:
+        pass
+    n = 8 * world
+    st = ddp.PeerMappedStates(n, "cpu")
+    ok = ok and st.world == world and st.rank == rank and st.n == n
+    ok = ok and bool((st.m == 0).all()) and bool((st.v == 0).all()) and bool((st.w == 7).all())
+    st.exchange_and_apply(Opt(), 1e-3)
+    kinds = [e[0] for e in log]
+    ok = ok and kinds == ["barrier", "launch", "barrier"]
+    launch = log[1]
+    ok = ok and launch[4] == rank and launch[5] == n and launch[6] == 1e-3
+    ok = ok and all(len(p) == world for p in launch[1:4])
+    ok = ok and len({tuple(launch[1]), tuple(launch[2]), tuple(launch[3])}) == 3
+    (Path(out_dir) / f"peer{rank}.json").write_text(json.dumps({"ok": bool(ok), "log": kinds}))
+    dist.destroy_process_group()
+
+
+def test_peer_mapped_states_protocol_with_stand_in_handles(tmp_path):
+    world = 2
+    port = _free_port()
+    mp.spawn(_peer_states_rank, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    for r in range(world):
+        res = json.loads((tmp_path / f"peer{r}.json").read_text())
+        assert res["ok"], res

@@ -102,6 +102,84 @@ def test_timeout_report_path_without_a_waiting_kernel():
     opt.close()
 
 
+@pytest.mark.parametrize("tokens,epilogue", [(256, 0), (2304, 0), (256, 1), (2304, 2)])
+def test_device_side_wait_runs_out_and_the_kernel_returns(tokens, epilogue):
+    """A wait inside the fused kernel that really expires, in the non-hanging form: the test
+    entry launches the normal kernel with a 1 ms limit on every wait and a producer that
+    never loads the last stage of the last tile.  The kernel must come back by itself (the
+    synchronise below returns), report a time-out with the wait and the tile, leave the
+    other tiles folded and the withheld tile untouched, and the same context must then pass
+    a normal call.  Both epilogue forms (256 tokens: staged, 2304: direct; and each forced the
+    other way)."""
+    import time
+    import adama_workloads as wl
+    d_in, d_out = 512, 768                      # 2 x 3 tiles; the withheld one is the last
+    opt = adama.AdamA()
+    opt.debug_set_wgrad_variant(epilogue=epilogue)
+    opt.begin_minibatch(1)
+    X = wl.small_integers((tokens, d_in), 2, torch.bfloat16, 1).cuda()
+    dY = wl.small_integers((tokens, d_out), 2, torch.bfloat16, 2).cuda()
+    m = torch.zeros(d_in, d_out, device="cuda")
+    v = torch.zeros(d_in, d_out, device="cuda")
+    t0 = time.perf_counter()
+    opt.debug_wgrad_expire_wait(X, dY, m, v, wait_limit_ns=1_000_000)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0       # limits of 1 ms (+20 ms of draining), not 2 s
+    with pytest.raises(adama.AdamAError) as e:
+        opt.sync_status()
+    assert e.value.status == Status.ERR_TIMEOUT
+    assert "wait" in str(e.value) and "tile" in str(e.value)
+    G = X.float().t() @ dY.float()              # small integers: exact in fp32
+    want = (1 - 0.9) * G
+    # the withheld work item is the launch's last: the bottom-right tile, or its right half
+    # when the launch issues its tiles as column halves
+    missing = (m == 0) & (G != 0)
+    rows = missing.any(dim=1).nonzero().flatten()
+    cols = missing.any(dim=0).nonzero().flatten()
+    assert int(rows.min()) >= 256 and int(cols.min()) in (512, 640)
+    done = torch.ones(d_in, d_out, dtype=torch.bool, device="cuda")
+    done[256:, int(cols.min()):] = False
+    assert torch.allclose(m[done], want[done], rtol=1e-6)
+    assert bool((m[~done] == 0).all()) and bool((v[~done] == 0).all())
+    opt.sync_status()                           # cleared by the report
+    m.zero_()
+    v.zero_()
+    opt.linear_wgrad_fold(X, dY, m, v)          # the context (and the GPU) are still usable
+    opt.sync_status()
+    assert torch.allclose(m, want, rtol=1e-6)
+    assert torch.allclose(v, (1 - 0.999) * G * G, rtol=1e-6)
+    opt.close()
+
+
+def test_expire_wait_entry_rejects_limits_out_of_range():
+    opt = adama.AdamA()
+    opt.begin_minibatch(1)
+    X = torch.zeros(64, 128, dtype=torch.bfloat16, device="cuda")
+    dY = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
+    m = torch.zeros(128, 256, device="cuda")
+    for limit in (0, 999, 2_000_000_000):
+        with pytest.raises(adama.AdamAError) as e:
+            opt.debug_wgrad_expire_wait(X, dY, m, m.clone(), wait_limit_ns=limit)
+        assert e.value.status == Status.ERR_INVALID_ARG
+    assert opt.launch_count == 0
+    opt.close()
+
+
+def test_setup_state_after_a_launch_on_device_0():
+    """Kernel attributes are remembered per device: after a fused launch on device 0 the
+    table says so for device 0 and for no other device."""
+    opt = adama.AdamA()
+    opt.begin_minibatch(1)
+    X = torch.zeros(64, 128, dtype=torch.bfloat16, device="cuda")
+    dY = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
+    m = torch.zeros(128, 256, device="cuda")
+    opt.linear_wgrad_fold(X, dY, m, m.clone())
+    opt.sync_status()
+    assert adama.debug_setup_state(0) == 3
+    assert adama.debug_setup_state(1) & 2 == 0 and adama.debug_setup_state(64) & 2 == 0
+    opt.close()
+
+
 def test_checkpoint_resume_is_bit_identical():
     """State = w, m, v (stored decayed after apply) + the step counter: a new context restored
     with set_step continues exactly as the uninterrupted run."""

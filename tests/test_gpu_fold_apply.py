@@ -11,7 +11,7 @@ import torch
 import adama_workloads as wl
 import paper_2305_19982_b200 as adama
 from oracle import AdamAOracle
-from parity import Guarded, f64, rel_l2
+from parity import Guarded, assert_close, f64, rel_l2
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-6
@@ -34,13 +34,13 @@ def _run_flat(cfg: wl.FlatConfig, n: int, steps: int, offset=0, g_offset=0):
             g.fill(grad.cuda())
             opt.fold(g.view, m.view, v.view)
             orc.fold(f64(grad))
-        assert rel_l2(f64(m.view), orc.m) <= TOL
-        assert rel_l2(f64(v.view), orc.v) <= TOL
+        assert_close(f64(m.view), orc.m, TOL, "m_t")
+        assert_close(f64(v.view), orc.v, TOL, "v_t")
         opt.apply(w.view, m.view, v.view, wl.LR)
         orc.update(wl.LR)
-        assert rel_l2(f64(w.view), orc.theta) <= TOL
-        assert rel_l2(f64(m.view), wl.BETA1 * orc.m) <= TOL
-        assert rel_l2(f64(v.view), wl.BETA2 * orc.v) <= TOL
+        assert_close(f64(w.view), orc.theta, TOL, "w")
+        assert_close(f64(m.view), wl.BETA1 * orc.m, TOL, "beta1*m")
+        assert_close(f64(v.view), wl.BETA2 * orc.v, TOL, "beta2*v")
         assert opt.step == orc.t == step + 1
     for b in (w, m, v, g):
         b.check()
@@ -112,7 +112,11 @@ def test_many_steps_decay_has_no_drift():
     relative, so a random walk of ~sqrt(800) * 4.8e-8 = 1.4e-6 is what fp32 state must show;
     the bound is twice that.  What must NOT appear is a bias: a plain fp32 beta2 (relative
     error 1.3e-8) would shift every element of v by about -1.3e-6 after 200 steps, which the
-    mean signed error (noise 1.4e-6/sqrt(n)) exposes."""
+    mean signed error (noise 1.4e-6/sqrt(n)) exposes.
+    The first moment forgets: with beta1 = 0.9 a rounding made k steps ago survives with weight
+    beta1^k, so its error is the geometric sum sqrt(4/(1-beta1^2)) = 4.6 roundings' worth,
+    2.2e-7 relative to the size of m, however many steps are run; the bound is twice that, and
+    a bias in its decay would show in w (below) long before it showed in m."""
     n, N, steps = 4096, 2, 200
     opt = adama.AdamA()
     w0 = wl.normal((n,), 0.02, torch.float32, 1)
@@ -132,6 +136,8 @@ def test_many_steps_decay_has_no_drift():
     assert rel_l2(f64(v), want_v) <= 2 * random_walk
     bias = float(np.mean((f64(v) - want_v) / want_v))
     assert abs(bias) <= 2e-7, bias
+    forgetful_walk = np.sqrt(4 / (1 - wl.BETA1 ** 2)) * 2.0 ** -24 / np.sqrt(3) * 1.4
+    assert rel_l2(f64(m), wl.BETA1 * orc.m) <= 2 * forgetful_walk
     assert rel_l2(f64(w), orc.theta) <= TOL
     opt.close()
 

@@ -13,7 +13,7 @@ import adama_workloads as wl
 import oracle
 import paper_2305_19982_b200 as adama
 from oracle import AdamAOracle
-from parity import SENTINEL, f64, rel_l2
+from parity import SENTINEL, assert_close, f64
 
 pytestmark = pytest.mark.gpu
 TOL_BF16 = 2e-3
@@ -30,11 +30,14 @@ def _draw(T, d_in, d_out, seed, integer=False):
     return X, dY
 
 
-def _full_parity(T, d_in, d_out, n_micro=2, steps=1, integer=False, pad=0, tol=None):
+def _full_parity(T, d_in, d_out, n_micro=2, steps=1, integer=False, pad=0, tol=None, variant=None):
     """Whole-matrix comparison; `pad` > 0 embeds X, dY, m, v in wider buffers (row pitch >
-    row length) whose extra columns hold a sentinel that must survive."""
+    row length) whose extra columns hold a sentinel that must survive.  `variant` pins the
+    kernel instance (adama_debug_set_wgrad_variant) instead of the automatic choice."""
     tol = tol if tol is not None else (TOL_EXACT if integer else TOL_BF16)
     opt = adama.AdamA()
+    if variant:
+        opt.debug_set_wgrad_variant(**variant)
     w0 = wl.normal((d_in, d_out), 0.02, torch.float32, 77)
     orc = AdamAOracle(f64(w0))
     up = lambda x, k: (x + k - 1) // k * k
@@ -59,15 +62,15 @@ def _full_parity(T, d_in, d_out, n_micro=2, steps=1, integer=False, pad=0, tol=N
             opt.linear_wgrad_fold(Xb[:, :d_in], Yb[:, :d_out], m, v)
             orc.fold_linear(f64(X), f64(dY))
         opt.sync_status()
-        assert rel_l2(f64(m), orc.m) <= tol
-        assert rel_l2(f64(v), orc.v) <= tol
+        assert_close(f64(m), orc.m, tol, "m_t")
+        assert_close(f64(v), orc.v, tol, "v_t")
         # apply works on contiguous buffers: use dense copies of the views
         mc, vc = m.contiguous(), v.contiguous()
         opt.apply(w, mc, vc, wl.LR)
         orc.update(wl.LR)
         m.copy_(mc)
         v.copy_(vc)
-        assert rel_l2(f64(w), orc.theta) <= tol
+        assert_close(f64(w), orc.theta, tol, "w", elementwise=integer or n_micro > 1 or step > 0)
     if pad:
         assert bool((mbuf[:, d_out:] == SENTINEL).all()) and bool((vbuf[:, d_out:] == SENTINEL).all())
     opt.close()
@@ -133,6 +136,48 @@ def test_more_tiles_than_sms():
     _full_parity(640, 2048, 4096, n_micro=1, integer=False)
 
 
+@pytest.mark.parametrize("T,d_in,d_out,why", [
+    (640, 2048, 4096, "128 full tiles on 74 CTA pairs: second accumulator stage, ring phase wrap"),
+    (128, 5120, 1024, "20 x 4 tiles: row index slowest, 6 left-over tiles issued as column halves"),
+    (192, 1024, 5120, "4 x 20 tiles: column index slowest, same split tail"),
+    (320, 1600, 1600, "layer of the GPT-2-XL-shaped stack: ragged last row and column tiles"),
+    (2112, 1600, 4800, "the same beyond the short-call limit, several k-blocks per ring wrap"),
+    (1100, 1664, 832, "short-call (staged) instance over more than one round of tiles"),
+])
+def test_whole_matrix_exact_beyond_one_round_of_tiles(T, d_in, d_out, why):
+    """Shapes that need more than one tile per CTA group, a split tail or either tile
+    numbering, with small-integer inputs (|x| <= 4: every product and every partial sum over
+    at most 2112 tokens is below 2^24, hence exact in fp32).  The whole matrix is compared
+    with the oracle at the fp32 fold tolerance, in the L2 norm and element by element, so one
+    wrong chunk, tile or accumulator stage cannot hide."""
+    _full_parity(T, d_in, d_out, n_micro=2, integer=True)
+
+
+@pytest.mark.parametrize("variant", [
+    dict(epilogue=1, epi_warps=4), dict(epilogue=1, epi_warps=8), dict(epilogue=2),
+    dict(box_loads=1), dict(no_pdl=1), dict(epilogue=2, box_loads=1, no_pdl=1)],
+    ids=lambda v: ",".join(f"{k}={x}" for k, x in v.items()))
+@pytest.mark.parametrize("T,d_in,d_out,pad", [(320, 300, 1000, 5), (2240, 512, 768, 0),
+                                              (192, 2560, 2048, 0)])
+def test_every_kernel_instance_on_every_kind_of_shape(variant, T, d_in, d_out, pad):
+    """The launch picks an epilogue form, a warp count and a load form from the shape; here each
+    is pinned in turn, on a ragged shape in padded buffers, on a shape that allows grouped
+    loads (both sides of the short-call limit) and on one with more tiles than CTA pairs, so
+    that no instance is only ever reached by the shapes that happen to select it.  Integer
+    inputs: exact contraction, fp32 fold tolerance."""
+    _full_parity(T, d_in, d_out, integer=True, pad=pad, variant=variant)
+
+
+def test_variant_entry_rejects_values_out_of_range():
+    opt = adama.AdamA()
+    for bad in (dict(epilogue=3), dict(epi_warps=6), dict(box_loads=2), dict(no_pdl=-1),
+                dict(tile_cols=48), dict(tile_cols=288)):
+        with pytest.raises(adama.AdamAError) as e:
+            opt.debug_set_wgrad_variant(**bad)
+        assert e.value.status == adama.Status.ERR_INVALID_ARG
+    opt.close()
+
+
 def test_long_contraction_phase_wraps():
     _full_parity(4096 + 48, 256, 512, n_micro=1)
 
@@ -171,12 +216,13 @@ def _sampled_parity(T, d_in, d_out, n_micro, steps, config, count=3000):
             opt.linear_wgrad_fold(X, dY, m, v)
             orc.fold(oracle.linear_wgrad_entries(f64(X), f64(dY), p, q))
         opt.sync_status()
-        assert rel_l2(f64(m.view(-1)[flat]), orc.m) <= TOL_BF16
-        assert rel_l2(f64(v.view(-1)[flat]), orc.v) <= TOL_BF16
+        assert_close(f64(m.view(-1)[flat]), orc.m, TOL_BF16, "m_t")
+        assert_close(f64(v.view(-1)[flat]), orc.v, TOL_BF16, "v_t")
         opt.apply(w, m, v, wl.LR)
         orc.update(wl.LR)
-        assert rel_l2(f64(w.view(-1)[flat]), orc.theta) <= TOL_BF16
-        assert rel_l2(f64(m.view(-1)[flat]), wl.BETA1 * orc.m) <= TOL_BF16
+        assert_close(f64(w.view(-1)[flat]), orc.theta, TOL_BF16, "w", elementwise=n_micro > 1 or step > 0)
+        assert_close(f64(m.view(-1)[flat]), wl.BETA1 * orc.m, TOL_BF16, "beta1*m")
+        assert_close(f64(v.view(-1)[flat]), wl.BETA2 * orc.v, TOL_BF16, "beta2*v")
     assert bool((v >= 0).all()) and bool(torch.isfinite(m).all()) and bool(torch.isfinite(w).all())
     opt.close()
 
