@@ -4,13 +4,17 @@
 //   m[p,q] += a*G[p,q];   v[p,q] += b*G[p,q]^2       (Algorithm 2, inner loop body)
 //
 // G lives only as an accumulator tile in tensor memory.  The epilogue issues the
-// coalesced 128-bit loads of the matching m and v chunk first, reads the accumulator
+// coalesced 128-bit loads of the matching m chunk first, reads the accumulator
 // chunk with tcgen05.ld while they are in flight, turns it from "one row per thread"
 // into "128 contiguous bytes per quarter-warp" through a swizzled shared-memory
-// buffer, and writes fma(a, G, m) and fma(b*G, G, v) back with 128-bit stores.
-// (Letting the L2 do the read-modify-write -- TMA reduce-add or red.global.add.v4 --
-// was measured first: the L2's reduction rate, about 2 TB/s of payload, stalled the
-// operand loads of the overlapped main loop; plain reads and writes do not.)
+// buffer, writes fma(a, G, m) back with 128-bit stores and hands (b*G)*G to the L2 as
+// a reduction into v (red.global.add.v4.f32).  What bounds the main loop is the SM's
+// inbound port from the L2 (about 118 GB/s per SM measured with TMA loads alone): a
+// 256x256 pair tile needs 512 bytes of operands per token and SM, and the m, v reads of
+// the overlapped epilogue come through the same port.  Sending v's half of the state
+// traffic as reductions takes it off that port (config-3 call 122 -> 117 us); sending
+// m's half too was measured slower (127 us): the L2's reduction rate then holds up the
+// operand loads.
 //
 // Persistent kernel, 192 or 320 threads per CTA, CTAs working in pairs (a cluster of two on
 // the two SMs of a TPC, tcgen05 cta_group::2): a pair owns a 256x256 output tile,
@@ -311,6 +315,13 @@ __device__ __forceinline__ void st_global_v4(float *p, float4 x) {
                  "f"(x.w)
                  : "memory");
 }
+// v += x as a reduction performed by the L2: the old value never enters the SM.  Every element
+// is touched by exactly one thread per call, so the result is as deterministic as a store.
+__device__ __forceinline__ void red_add_v4(float *p, float4 x) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z),
+                 "f"(x.w)
+                 : "memory");
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, float x, float y, float z, float w) {
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z),
                  "f"(w)
@@ -600,83 +611,114 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         // ---------------- staged epilogue, streaming side: shared-memory tile -> m, v ----------------
         // A warp owns 16 rows of the CTA's 128; the tile comes in parts of PART_COLS columns, so
         // that one part is folded while the drain warps copy the next.  A warp instruction covers
-        // 32/LPR rows x PART_COLS*4 contiguous bytes; eight such loads of m and of v are in flight
-        // per thread.
+        // 32/LPR rows x PART_COLS*4 contiguous bytes.  m is read, folded and written back; v takes
+        // its increment through an L2 reduction, so only half of the state traffic enters the SM.
+        // The eight m loads of the NEXT part (or of the next tile's first part) are issued before
+        // the current part is folded: the loads never drain between parts.
         const int sw_id = warp - (2 + STAGED_DRAIN_WARPS);
         const uint32_t gbuf = base + G::SMEM_EPI_OFF;
         constexpr int LPR = PART_COLS / 4;   // lanes per row: a warp instruction covers 32 / LPR rows
         constexpr int RPI = 32 / LPR;
         constexpr int PITCH = PART_COLS * 4;  // bytes per row of a part buffer
+        static_assert(8 * RPI == 16, "a warp's 16 rows of a part are one batch of eight loads");
         const int sub = lane / LPR, cl = lane % LPR;
+        const int lrow0 = sw_id * 16 + sub;  // this thread's first row of the CTA's 128
         bool ok = true;
         uint32_t use_bits = 0;    // bit k: parity of how often part buffer k has been used
         grid_dependency_wait();   // m and v may still be written by the previous call
-        for (int tile = group; tile < num_items && ok; tile += num_groups) {
+
+        struct Part {
+            float *pm, *pv;
+            int row_first, gcol;
+            bool col_vec;
+        };
+        auto part_at = [&](int tile, int part_i) {
             const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
-            const int row_base = wi.m0 + (int)rank * G::ROWS_PER_CTA;
-            for (int part_i = 0; part_i < wi.width / PART_COLS; ++part_i) {
-                if (!ok) continue;
-                const int k = part_i & 1;
-                ok = mbar_wait(smem_u32(&bars->g_full[k]), (use_bits >> k) & 1u, abort_flag, wait_limit_ns);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) {
-                    if (lane == 0) record_timeout(status, bars, 7, (unsigned)tile);
-                    continue;
-                }
-                use_bits ^= 1u << k;
-                const uint32_t pbuf = gbuf + (uint32_t)k * PART_BYTES;
-                const int gcol = wi.n0 + part_i * PART_COLS + cl * 4;
-                const bool col_vec = gcol + 4 <= d_out;  // whole group of four columns inside
-                for (int rb = 0; rb < 16; rb += 8 * RPI) {
-                    const int lrow0 = sw_id * 16 + rb + sub;  // this thread's first row of the batch
-                    float *pm = m_out + (long long)(row_base + lrow0) * ldmv + gcol;
-                    float *pv = v_out + (long long)(row_base + lrow0) * ldmv + gcol;
-                    float4 mm[8], vv[8];
-                    if (col_vec) {
+            Part u;
+            u.row_first = wi.m0 + (int)rank * G::ROWS_PER_CTA + lrow0;
+            u.gcol = wi.n0 + part_i * PART_COLS + cl * 4;
+            u.col_vec = u.gcol + 4 <= d_out;  // whole group of four columns inside
+            u.pm = m_out + (long long)u.row_first * ldmv + u.gcol;
+            u.pv = v_out + (long long)u.row_first * ldmv + u.gcol;
+            return u;
+        };
+        auto load_m = [&](const Part &u, float4(&mm)[8]) {
+            if (u.col_vec) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (row_base + lrow0 + i * RPI < d_in) {
-                                mm[i] = ld_global_v4_stream(pm + (long long)(i * RPI) * ldmv);
-                                vv[i] = ld_global_v4_stream(pv + (long long)(i * RPI) * ldmv);
-                            }
+                for (int i = 0; i < 8; ++i)
+                    if (u.row_first + i * RPI < d_in)
+                        mm[i] = ld_global_v4_stream(u.pm + (long long)(i * RPI) * ldmv);
+            }
+        };
+        // waits for part buffer k to hold the part, folds it, hands the buffer back
+        auto fold_part = [&](const Part &u, float4(&mm)[8], int k, int tile) {
+            ok = mbar_wait(smem_u32(&bars->g_full[k]), (use_bits >> k) & 1u, abort_flag, wait_limit_ns);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) record_timeout(status, bars, 7, (unsigned)tile);
+                return;
+            }
+            use_bits ^= 1u << k;
+            const uint32_t pbuf = gbuf + (uint32_t)k * PART_BYTES;
+            if (u.col_vec) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (row_base + lrow0 + i * RPI < d_in) {
-                                const int lrow = lrow0 + i * RPI;
-                                const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
-                                                              (uint32_t)((cl ^ (lrow & 7)) << 4));
-                                float4 &x = mm[i], &y = vv[i];
-                                x.x = fmaf(a, g.x, x.x);
-                                x.y = fmaf(a, g.y, x.y);
-                                x.z = fmaf(a, g.z, x.z);
-                                x.w = fmaf(a, g.w, x.w);
-                                y.x = fmaf(b * g.x, g.x, y.x);
-                                y.y = fmaf(b * g.y, g.y, y.y);
-                                y.z = fmaf(b * g.z, g.z, y.z);
-                                y.w = fmaf(b * g.w, g.w, y.w);
-                                st_global_v4(pm + (long long)(i * RPI) * ldmv, x);
-                                st_global_v4(pv + (long long)(i * RPI) * ldmv, y);
-                            }
-                    } else if (gcol < d_out) {
-                        // last, partial group of four columns: element-wise
-                        for (int i = 0; i < 8; ++i) {
-                            const int lrow = lrow0 + i * RPI;
-                            if (row_base + lrow >= d_in) break;
-                            const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
-                                                          (uint32_t)((cl ^ (lrow & 7)) << 4));
-                            const float ge[4] = {g.x, g.y, g.z, g.w};
-                            for (int e = 0; e < 4; ++e)
-                                if (gcol + e < d_out) {
-                                    float *qm = pm + (long long)(i * RPI) * ldmv + e;
-                                    float *qv = pv + (long long)(i * RPI) * ldmv + e;
-                                    *qm = fmaf(a, ge[e], *qm);
-                                    *qv = fmaf(b * ge[e], ge[e], *qv);
-                                }
-                        }
+                for (int i = 0; i < 8; ++i)
+                    if (u.row_first + i * RPI < d_in) {
+                        const int lrow = lrow0 + i * RPI;
+                        const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
+                                                      (uint32_t)((cl ^ (lrow & 7)) << 4));
+                        float4 &x = mm[i];
+                        x.x = fmaf(a, g.x, x.x);
+                        x.y = fmaf(a, g.y, x.y);
+                        x.z = fmaf(a, g.z, x.z);
+                        x.w = fmaf(a, g.w, x.w);
+                        st_global_v4(u.pm + (long long)(i * RPI) * ldmv, x);
+                        red_add_v4(u.pv + (long long)(i * RPI) * ldmv,
+                                   make_float4((b * g.x) * g.x, (b * g.y) * g.y, (b * g.z) * g.z,
+                                               (b * g.w) * g.w));
                     }
+            } else if (u.gcol < d_out) {
+                // last, partial group of four columns: element-wise
+                for (int i = 0; i < 8; ++i) {
+                    const int lrow = lrow0 + i * RPI;
+                    if (u.row_first + i * RPI >= d_in) break;
+                    const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
+                                                  (uint32_t)((cl ^ (lrow & 7)) << 4));
+                    const float ge[4] = {g.x, g.y, g.z, g.w};
+                    for (int e = 0; e < 4; ++e)
+                        if (u.gcol + e < d_out) {
+                            float *qm = u.pm + (long long)(i * RPI) * ldmv + e;
+                            float *qv = u.pv + (long long)(i * RPI) * ldmv + e;
+                            *qm = fmaf(a, ge[e], *qm);
+                            *qv += (b * ge[e]) * ge[e];
+                        }
                 }
-                __syncwarp();  // every lane has read its share of this part
-                if (lane == 0) mbar_arrive(smem_u32(&bars->g_empty[k]));
+            }
+            __syncwarp();  // every lane has read its share of this part
+            if (lane == 0) mbar_arrive(smem_u32(&bars->g_empty[k]));
+        };
+
+        if (group < num_items) {
+            float4 m_a[8], m_b[8];
+            Part u_a = part_at(group, 0), u_b = u_a;
+            load_m(u_a, m_a);
+            for (int tile = group; tile < num_items && ok; tile += num_groups) {
+                // parts per tile: 4 (full tile) or 2 (half tile); part i lives in buffer i & 1
+                const int nparts = work_item(tile, split_from, tiles_m, tiles_n).width / PART_COLS;
+                for (int part_i = 0; part_i < nparts && ok; part_i += 2) {
+                    u_b = part_at(tile, part_i + 1);
+                    load_m(u_b, m_b);
+                    fold_part(u_a, m_a, 0, tile);
+                    if (!ok) break;
+                    if (part_i + 2 < nparts) {
+                        u_a = part_at(tile, part_i + 2);
+                        load_m(u_a, m_a);
+                    } else if (tile + num_groups < num_items) {
+                        u_a = part_at(tile + num_groups, 0);
+                        load_m(u_a, m_a);
+                    }
+                    fold_part(u_b, m_b, 1, tile);
+                }
             }
         }
     } else if (warp >= first_bias_warp) {
@@ -820,7 +862,12 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 }
             }
         } else {
-        // ---------------- epilogue: m = fma(a, G, m), v = fma(b*G, G, v) ----------------
+        // ---------------- epilogue: m = fma(a, G, m), v += (b*G)*G ----------------
+        // m is read, folded and written back by the SM; v takes its increment through an L2
+        // reduction (red.global.add), so that only half of the state traffic enters the SM:
+        // the SM's inbound port, which also carries the operand tiles, is what bounds the
+        // main loop that this epilogue overlaps.  The m loads of a tile's first chunk are issued
+        // before the wait for its accumulator.
         const int q = warp & 3;            // TMEM lane quarter this warp may read
         const int part = (warp - 2) >> 2;  // which part of the tile's columns it handles
         const int col_split = epi_warps / 4;  // 1 or 2 warps per lane quarter
@@ -835,12 +882,84 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         bool ok = true;
         int it = 0;
         grid_dependency_wait();  // m and v may still be written by the previous call
+
+        // one 32 x 32 chunk of the tile: geometry, m loads, fold
+        struct Chunk {
+            long long off0;
+            int col0;
+            bool inside, interior;
+        };
+        auto chunk_at = [&](const WorkItem &wi, int row0, int c) {
+            Chunk ch;
+            ch.col0 = wi.n0 + c * EPI_COLS;
+            ch.inside = row0 < d_in && ch.col0 < d_out;
+            ch.interior = row0 + EPI_ROWS <= d_in && ch.col0 + EPI_COLS <= d_out;
+            ch.off0 = (long long)(row0 + sub_row) * ldmv + ch.col0 + c4 * 4;
+            return ch;
+        };
+        auto load_m = [&](const Chunk &ch, float4(&mm)[8]) {
+            if (ch.interior) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    mm[i] = ld_global_v4_stream(m_out + ch.off0 + (long long)i * 4 * ldmv);
+            }
+        };
+        auto fold_chunk = [&](const Chunk &ch, float4(&mm)[8], uint32_t taddr, int row0) {
+            if (!ch.inside) return;  // chunks wholly outside the matrix are skipped
+            uint32_t r[32];
+            tc_ld_32x32(taddr, r);
+            tc_wait_ld();
+            __syncwarp();  // the previous chunk has been read out of the buffer
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                st_shared_v4(sm_g + row_off + ((((uint32_t)j) ^ sw) << 4),
+                             __uint_as_float(r[4 * j + 0]), __uint_as_float(r[4 * j + 1]),
+                             __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+            __syncwarp();
+            if (ch.interior) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int row = i * 4 + sub_row;
+                    const float4 g = ld_shared_v4(sm_g + (uint32_t)row * 128u +
+                                                  (uint32_t)((c4 ^ (row & 7)) << 4));
+                    mm[i].x = fmaf(a, g.x, mm[i].x);
+                    mm[i].y = fmaf(a, g.y, mm[i].y);
+                    mm[i].z = fmaf(a, g.z, mm[i].z);
+                    mm[i].w = fmaf(a, g.w, mm[i].w);
+                    st_global_v4(m_out + ch.off0 + (long long)i * 4 * ldmv, mm[i]);
+                    red_add_v4(v_out + ch.off0 + (long long)i * 4 * ldmv,
+                               make_float4((b * g.x) * g.x, (b * g.y) * g.y, (b * g.z) * g.z,
+                                           (b * g.w) * g.w));
+                }
+            } else {
+                // ragged edge of the matrix: element-wise, bounds-checked
+                for (int i = 0; i < 8; ++i) {
+                    const int row = i * 4 + sub_row;
+                    if (row0 + row >= d_in) continue;
+                    const float4 g = ld_shared_v4(sm_g + (uint32_t)row * 128u +
+                                                  (uint32_t)((c4 ^ (row & 7)) << 4));
+                    const float ge[4] = {g.x, g.y, g.z, g.w};
+                    float *pm = m_out + ch.off0 + (long long)i * 4 * ldmv;
+                    float *pv = v_out + ch.off0 + (long long)i * 4 * ldmv;
+                    for (int e = 0; e < 4; ++e)
+                        if (ch.col0 + c4 * 4 + e < d_out) {
+                            pm[e] = fmaf(a, ge[e], pm[e]);
+                            pv[e] += (b * ge[e]) * ge[e];
+                        }
+                }
+            }
+        };
+
         for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
             const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
             const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
             const int chunks = wi.width / (col_split * EPI_COLS);  // chunks per warp
+            const int c_first = part * chunks;
+            float4 mm[8];
+            Chunk ch = chunk_at(wi, row0, c_first);
+            load_m(ch, mm);  // in flight while the tile's main loop still runs
             ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag, wait_limit_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -848,68 +967,14 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                 break;
             }
             tc_fence_after();
-            if (row0 < d_in) {
-                const uint32_t taddr0 =
-                    tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
-                for (int cc = 0; cc < chunks; ++cc) {
-                    const int c = part * chunks + cc;
-                    const int col0 = wi.n0 + c * EPI_COLS;
-                    if (col0 >= d_out) break;  // chunks wholly outside the matrix are skipped
-                    const long long off0 = (long long)(row0 + sub_row) * ldmv + col0 + c4 * 4;
-                    const bool interior = row0 + EPI_ROWS <= d_in && col0 + EPI_COLS <= d_out;
-                    float4 mm[8], vv[8];
-                    if (interior) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            mm[i] = ld_global_v4_stream(m_out + off0 + (long long)i * 4 * ldmv);
-                            vv[i] = ld_global_v4_stream(v_out + off0 + (long long)i * 4 * ldmv);
-                        }
-                    }
-                    uint32_t r[32];
-                    tc_ld_32x32(taddr0 + (uint32_t)(c * EPI_COLS), r);
-                    tc_wait_ld();
-                    __syncwarp();  // the previous chunk has been read out of the buffer
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        st_shared_v4(sm_g + row_off + ((((uint32_t)j) ^ sw) << 4),
-                                     __uint_as_float(r[4 * j + 0]), __uint_as_float(r[4 * j + 1]),
-                                     __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-                    __syncwarp();
-                    if (interior) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int row = i * 4 + sub_row;
-                            const float4 g = ld_shared_v4(sm_g + (uint32_t)row * 128u +
-                                                          (uint32_t)((c4 ^ (row & 7)) << 4));
-                            mm[i].x = fmaf(a, g.x, mm[i].x);
-                            mm[i].y = fmaf(a, g.y, mm[i].y);
-                            mm[i].z = fmaf(a, g.z, mm[i].z);
-                            mm[i].w = fmaf(a, g.w, mm[i].w);
-                            vv[i].x = fmaf(b * g.x, g.x, vv[i].x);
-                            vv[i].y = fmaf(b * g.y, g.y, vv[i].y);
-                            vv[i].z = fmaf(b * g.z, g.z, vv[i].z);
-                            vv[i].w = fmaf(b * g.w, g.w, vv[i].w);
-                            st_global_v4(m_out + off0 + (long long)i * 4 * ldmv, mm[i]);
-                            st_global_v4(v_out + off0 + (long long)i * 4 * ldmv, vv[i]);
-                        }
-                    } else {
-                        // ragged edge of the matrix: element-wise, bounds-checked
-                        for (int i = 0; i < 8; ++i) {
-                            const int row = i * 4 + sub_row;
-                            if (row0 + row >= d_in) continue;
-                            const float4 g = ld_shared_v4(sm_g + (uint32_t)row * 128u +
-                                                          (uint32_t)((c4 ^ (row & 7)) << 4));
-                            const float ge[4] = {g.x, g.y, g.z, g.w};
-                            float *pm = m_out + off0 + (long long)i * 4 * ldmv;
-                            float *pv = v_out + off0 + (long long)i * 4 * ldmv;
-                            for (int e = 0; e < 4; ++e)
-                                if (col0 + c4 * 4 + e < d_out) {
-                                    pm[e] = fmaf(a, ge[e], pm[e]);
-                                    pv[e] = fmaf(b * ge[e], ge[e], pv[e]);
-                                }
-                        }
-                    }
+            const uint32_t taddr0 =
+                tmem_base + ((uint32_t)(q * EPI_ROWS) << 16) + (uint32_t)(as * BN);
+            for (int cc = 0; cc < chunks; ++cc) {
+                if (cc > 0) {
+                    ch = chunk_at(wi, row0, c_first + cc);
+                    load_m(ch, mm);
                 }
+                fold_chunk(ch, mm, taddr0 + (uint32_t)((c_first + cc) * EPI_COLS), row0);
             }
             // accumulator stage may now be overwritten by the pair's MMA warp
             tc_fence_before();
