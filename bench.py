@@ -403,10 +403,15 @@ def run_ours(args):
     torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_stacks:
         # the two layer-stack workloads in their stated configuration, 2 mini-batches each
-        stacks = {"gpt2xl": measure_stack("gpt2xl", 2, 1, dev_index=local)}
+        # ("_per_block": the linears of a transformer block folded by one grouped launch)
+        stacks = {"gpt2xl": measure_stack("gpt2xl", 2, 1, dev_index=local),
+                  "gpt2xl_per_block": measure_stack("gpt2xl", 2, 1, dev_index=local,
+                                                    with_gemm_pipeline=False, layers_per_launch=4)}
         free, _ = torch.cuda.mem_get_info()
         if free >= 100 * (1 << 30):
             stacks["llama7b"] = measure_stack("llama7b", 2, 1, dev_index=local)
+            stacks["llama7b_per_block"] = measure_stack("llama7b", 2, 1, dev_index=local,
+                                                        with_gemm_pipeline=False, layers_per_launch=7)
         else:
             stacks["llama7b"] = {"skipped": f"needs ~90 GB of free device memory, {free >> 30} GiB free"}
     if rank == 0:
@@ -581,11 +586,14 @@ def materialised_minibatch(stack, opt, n_micro, lr, inputs):
     stack.apply(opt, lr)
 
 
-def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, dev_index=0):
+def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, dev_index=0,
+                  layers_per_launch=1):
     """GPT-2-XL- / Llama-7B-shaped stack, one mini-batch per step in the workload's own
     configuration (N = 8 / 16 micro-batches of 4096 tokens, layers back to front, fused
     weight-gradient fold per layer, one apply): time, TFLOP/s of the whole mini-batch, clocks,
-    peak device memory without a gradient buffer, with a per-layer one and with a whole-model one."""
+    peak device memory without a gradient buffer, with a per-layer one and with a whole-model one.
+    layers_per_launch > 1: that many consecutive layers (a transformer block's linears) are folded
+    by one grouped launch, their X, dY released together after it."""
     import paper_2305_19982_b200 as adama
     from paper_2305_19982_b200.stack import gpt2xl_stack, llama7b_stack
 
@@ -610,7 +618,7 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
         return pool_x[spec.d_in][(i + j) & 1], pool_y[spec.d_out][(i + j) & 1]
 
     for _ in range(max(1, warmup)):
-        stack.minibatch(opt, n_micro, wl.LR, pooled)
+        stack.minibatch(opt, n_micro, wl.LR, pooled, layers_per_launch)
     torch.cuda.synchronize()
     sampler = ClockSampler(physical_gpu_index(dev_index))
     sampler.start()
@@ -619,7 +627,7 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
     stop = torch.cuda.Event(enable_timing=True)
     start.record()
     for _ in range(steps):
-        stack.minibatch(opt, n_micro, wl.LR, pooled)
+        stack.minibatch(opt, n_micro, wl.LR, pooled, layers_per_launch)
     stop.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -653,7 +661,7 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
         torch.cuda.synchronize()
         torch.cuda.reset_peak_memory_stats(dev)
         if mode == "none":
-            stack.minibatch(opt, 1, wl.LR, fresh)
+            stack.minibatch(opt, 1, wl.LR, fresh, layers_per_launch)
         else:
             materialised_minibatch(stack, opt, 1, wl.LR, fresh)
         torch.cuda.synchronize()
@@ -664,7 +672,7 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
     out = {
         "workload": kind, "biases": bool(stack.biases), "layers": len(stack.layers),
         "params": stack.n_params, "tokens_per_micro_batch": tokens, "n_micro": n_micro,
-        "steps": steps, "ms_per_minibatch": ms, "TFLOPps": tf,
+        "layers_per_launch": layers_per_launch, "steps": steps, "ms_per_minibatch": ms, "TFLOPps": tf,
         "frac_of_sustained_bf16": tf / pk["bf16_tflops_sustained"],
         "frac_of_burst_bf16": tf / pk["bf16_tflops"], "peak_source": pk["source"],
         "gpu_launches": int(launches), "clocks": clocks,
@@ -688,7 +696,8 @@ def run_stack(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(0)
-    r = measure_stack(args.workload, args.steps, min(args.warmup, 2), biases=args.biases)
+    r = measure_stack(args.workload, args.steps, min(args.warmup, 2), biases=args.biases,
+                      layers_per_launch=args.layers_per_launch)
     pk = peaks()
     line = {
         "metric": "adama_wgrad_fold_stack_TFLOPps", "value": r["TFLOPps"], "unit": "TFLOP/s", "n_gpus": 1,
@@ -697,7 +706,8 @@ def run_stack(args):
         "dtype": "bf16 inputs, f32 accumulate and state", "data": "synthetic",
         "config": {"workload": args.workload, "biases": r["biases"], "layers": r["layers"],
                    "params": r["params"], "tokens_per_micro_batch": r["tokens_per_micro_batch"],
-                   "n_micro": r["n_micro"], "l2": "inputs larger than L2, no flush"},
+                   "n_micro": r["n_micro"], "layers_per_launch": r["layers_per_launch"],
+                   "l2": "inputs larger than L2, no flush"},
         "roofline": {"kernel": "wgrad_fold_kernel", "bound": "tensor", "achieved": r["TFLOPps"],
                      "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": r["frac_of_sustained_bf16"], "frac_of_burst": r["frac_of_burst_bf16"],
@@ -1082,6 +1092,9 @@ def main():
                          "timed step (none = independent replicas; allreduce = Section 3.3's state "
                          "all-reduce; sharded = reduce-scatter of the states, all-gather of the weights)")
     ap.add_argument("--backend", default="gloo", help="launch_check only: process-group backend")
+    ap.add_argument("--layers-per-launch", type=int, default=1,
+                    help="gpt2xl / llama7b workloads: consecutive layers folded by one grouped launch "
+                         "(1 = one call per layer; 4 / 7 = one call per transformer block)")
     ap.add_argument("--no-stacks", action="store_true",
                     help="skip the two layer-stack workloads of the default line (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -147,6 +147,36 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
                                                int64_t ldy, float *m, float *v, int64_t ldmv,
                                                void *cuda_stream);
 
+/* adama_linear_wgrad_fold for several layers in as few launches as possible (at most 8 layers per
+ * launch), e.g. the linear layers of one transformer block whose (X, dY) pairs backward has
+ * produced.  Per layer it computes exactly what adama_linear_wgrad_fold (or, where m_bias and
+ * v_bias are given, adama_linear_wgrad_bias_fold) computes, bit for bit: Algorithm 2's inner
+ * loop body for layer j, for the `count` layers in the order given.  What changes is the
+ * schedule: the layers' tiles form one work list, so the CTA pairs that a layer's last round
+ * of tiles leaves idle start on the next layer, the epilogue of a layer's last tile overlaps
+ * the next layer's first main loop, and kernel set-up, pipeline fill and the final exposed
+ * epilogue are paid once per launch instead of once per layer.  The price is that the layers'
+ * X and dY must all be alive until the launch has run (they can be released one launch later
+ * than with per-layer calls; m, v and the weight gradient are unaffected: there still is no
+ * gradient buffer).  The layers must not share m or v storage.
+ *   items : `count` descriptions in HOST memory, read before the call returns; per item the
+ *           arguments of adama_linear_wgrad_fold, plus m_bias / v_bias (both null or both set).
+ * Items with tokens == 0 are skipped.  Errors: as adama_linear_wgrad_fold, reported for the
+ * first offending item before anything is launched. */
+typedef struct adama_linear_item {
+    const void *X;
+    const void *dY;
+    int tokens, d_in, d_out;
+    int64_t ldx, ldy;
+    float *m;
+    float *v;
+    int64_t ldmv;
+    float *m_bias; /* may be null (then v_bias must be null too) */
+    float *v_bias;
+} adama_linear_item;
+ADAMA_API adama_status adama_linear_wgrad_fold_multi(adama_ctx *ctx, const adama_linear_item *items,
+                                                     int count, void *cuda_stream);
+
 /* adama_linear_wgrad_fold that also folds the layer's bias gradient, the column sums of dY,
  *     g[q] = sum_{tau < tokens} dY[tau,q],   m_bias[q] += a*g[q],   v_bias[q] += b*g[q]^2
  * (Algorithm 2, inner loop body, for the bias of the same layer) in the same launch: two

@@ -19,7 +19,7 @@ EXPORTED_SYMBOLS = [
     "adama_init", "adama_destroy", "adama_begin_minibatch", "adama_fold",
     "adama_linear_wgrad_fold", "adama_linear_wgrad_bias_fold", "adama_apply", "adama_apply_bf16_copy", "adama_apply_allreduced", "adama_apply_sharded", "adama_apply_sharded_peers", "adama_fold_multi", "adama_apply_multi", "adama_bias_grad_fold",
     "adama_fold_host", "adama_linear_wgrad_fold_host",
-    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_sgdm_fold", "adama_sgdm_apply",
+    "adama_apply_to_host", "adama_linear_wgrad_fold_noalloc", "adama_linear_wgrad_fold_multi", "adama_sgdm_fold", "adama_sgdm_apply",
     "adama_coefficient_stats", "adama_get_step", "adama_set_step", "adama_get_n_micro", "adama_set_weight_decay",
     "adama_sync_status", "adama_debug_set_status", "adama_debug_wgrad_expire_wait",
     "adama_debug_set_wgrad_variant", "adama_debug_setup_state", "adama_last_error", "adama_launch_count", "adama_host_constants",
@@ -47,6 +47,13 @@ class AdamAError(RuntimeError):
     def __init__(self, status: int, message: str):
         self.status = Status(status)
         super().__init__(f"{self.status.name}: {message}")
+
+
+class _LinearItem(ctypes.Structure):
+    _fields_ = [("X", ctypes.c_void_p), ("dY", ctypes.c_void_p), ("tokens", ctypes.c_int),
+                ("d_in", ctypes.c_int), ("d_out", ctypes.c_int), ("ldx", ctypes.c_int64),
+                ("ldy", ctypes.c_int64), ("m", ctypes.c_void_p), ("v", ctypes.c_void_p),
+                ("ldmv", ctypes.c_int64), ("m_bias", ctypes.c_void_p), ("v_bias", ctypes.c_void_p)]
 
 
 class _Config(ctypes.Structure):
@@ -87,6 +94,7 @@ def load_library() -> ctypes.CDLL:
     L.adama_fold.argtypes = [vp, vp, ci, vp, vp, sz, vp]
     L.adama_linear_wgrad_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp]
     L.adama_linear_wgrad_bias_fold.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64, vp, vp, vp]
+    L.adama_linear_wgrad_fold_multi.argtypes = [vp, ctypes.POINTER(_LinearItem), ci, vp]
     L.adama_apply.argtypes = [vp, vp, vp, vp, sz, dbl, vp]
     L.adama_apply_bf16_copy.argtypes = [vp, vp, vp, vp, vp, sz, dbl, vp]
     L.adama_apply_allreduced.argtypes = [vp, vp, vp, vp, sz, dbl, ci, vp]
@@ -273,6 +281,39 @@ class AdamA:
             self._h, _dev_ptr(X, torch.bfloat16, "X"), _dev_ptr(dY, torch.bfloat16, "dY"),
             tokens, d_in, d_out, ldx, ldy, _dev_ptr(m, torch.float32, "m"),
             _dev_ptr(v, torch.float32, "v"), ldmv, _stream_ptr(self.device)))
+
+    def linear_wgrad_fold_multi(self, layers) -> None:
+        """adama_linear_wgrad_fold_multi: `layers` is a sequence of (X, dY, m, v) or
+        (X, dY, m, v, m_bias, v_bias) tuples, tensors as for linear_wgrad_fold; they are folded
+        in the given order by as few launches as possible.  Keep X and dY alive until the
+        stream has run the call."""
+        arr = (_LinearItem * len(layers))()
+        for it, layer in zip(arr, layers):
+            X, dY, m, v = layer[:4]
+            mb, vb = (layer[4], layer[5]) if len(layer) > 4 else (None, None)
+            if X.dim() != 2 or dY.dim() != 2 or m.dim() != 2 or v.dim() != 2:
+                raise ValueError("linear_wgrad_fold_multi takes 2-D tensors")
+            tokens, d_in = X.shape
+            d_out = dY.shape[1]
+            if dY.shape[0] != tokens or tuple(m.shape) != (d_in, d_out) or tuple(v.shape) != (d_in, d_out):
+                raise ValueError("shapes must be X [T, d_in], dY [T, d_out], m, v [d_in, d_out]")
+            for name, t in (("X", X), ("dY", dY), ("m", m), ("v", v)):
+                if t.shape[1] > 1 and t.stride(1) != 1:
+                    raise ValueError(f"{name} must have unit stride in its last dimension")
+            if m.stride(0) != v.stride(0):
+                raise ValueError("m and v must share one row pitch")
+            it.X, it.dY = _dev_ptr(X, torch.bfloat16, "X"), _dev_ptr(dY, torch.bfloat16, "dY")
+            it.tokens, it.d_in, it.d_out = tokens, d_in, d_out
+            it.ldx = X.stride(0) if tokens > 1 else max(d_in, X.stride(0))
+            it.ldy = dY.stride(0) if tokens > 1 else max(d_out, dY.stride(0))
+            it.m, it.v = _dev_ptr(m, torch.float32, "m"), _dev_ptr(v, torch.float32, "v")
+            it.ldmv = m.stride(0) if d_in > 1 else max(d_out, m.stride(0))
+            if mb is not None:
+                if mb.numel() != d_out or vb.numel() != d_out or not (mb.is_contiguous() and vb.is_contiguous()):
+                    raise ValueError("m_bias, v_bias must be contiguous with d_out elements")
+                it.m_bias, it.v_bias = _dev_ptr(mb, torch.float32, "m_bias"), _dev_ptr(vb, torch.float32, "v_bias")
+        self._check(self._L.adama_linear_wgrad_fold_multi(self._h, arr, len(layers),
+                                                          _stream_ptr(self.device)))
 
     def apply(self, w: torch.Tensor, m: torch.Tensor, v: torch.Tensor, lr: float) -> None:
         if not (w.is_contiguous() and m.is_contiguous() and v.is_contiguous()):

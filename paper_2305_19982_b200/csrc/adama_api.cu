@@ -296,6 +296,58 @@ adama_status adama_linear_wgrad_bias_fold(adama_ctx *ctx, const void *X, const v
                       cuda_stream);
 }
 
+adama_status adama_linear_wgrad_fold_multi(adama_ctx *ctx, const adama_linear_item *items, int count,
+                                           void *cuda_stream) {
+    if (!ctx) return ADAMA_ERR_INVALID_ARG;
+    if (count < 0 || (count > 0 && !items))
+        return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold_multi: null list or negative count");
+    for (int i = 0; i < count; ++i) {
+        const adama_linear_item &it = items[i];
+        adama_status st = check_wgrad_args(ctx, it.X, it.dY, it.tokens, it.d_in, it.d_out, it.ldx,
+                                           it.ldy, it.m, it.v, it.ldmv);
+        if (st != ADAMA_OK) return st;
+        if ((it.m_bias == nullptr) != (it.v_bias == nullptr))
+            return fail(ctx, ADAMA_ERR_INVALID_ARG, "wgrad_fold_multi: m_bias and v_bias go together");
+        if (!aligned_to(it.m_bias, 4) || !aligned_to(it.v_bias, 4))
+            return fail(ctx, ADAMA_ERR_MISALIGNED, "wgrad_fold_multi: bias moments not aligned to 4 bytes");
+    }
+    DeviceGuard guard(ctx->cfg.device);
+    adama::WgradArgs batch[adama::kMaxWgradLayers];
+    int k = 0;
+    for (int i = 0; i <= count; ++i) {
+        if ((i == count || k == adama::kMaxWgradLayers) && k > 0) {
+            const char *msg = "wgrad_fold_multi";
+            cudaError_t e = adama::launch_wgrad_fold_multi(batch, k, &msg);
+            if (e != cudaSuccess) return cuda_fail(ctx, msg, e);
+            ctx->launches += 1;
+            k = 0;
+        }
+        if (i == count) break;
+        const adama_linear_item &it = items[i];
+        if (it.tokens == 0) continue;  // empty sum: nothing to add
+        adama::WgradArgs &a = batch[k++];
+        a = adama::WgradArgs();
+        a.X = it.X;
+        a.dY = it.dY;
+        a.tokens = it.tokens;
+        a.d_in = it.d_in;
+        a.d_out = it.d_out;
+        a.ldx = it.ldx;
+        a.ldy = it.ldy;
+        a.ldmv = it.ldmv;
+        a.m = it.m;
+        a.v = it.v;
+        a.c = ctx->fold_c;
+        a.status = ctx->status_dev;
+        a.sm_count = ctx->sm_count;
+        a.stream = static_cast<cudaStream_t>(cuda_stream);
+        a.bias_m = it.m_bias;
+        a.bias_v = it.v_bias;
+        a.variant = ctx->variant;
+    }
+    return ADAMA_OK;
+}
+
 static adama_status apply_impl(adama_ctx *ctx, float *w, float *m, float *v, size_t n, double lr,
                                int world, bool sharded, void *cuda_stream,
                                void *w_bf16_out = nullptr) {

@@ -122,6 +122,10 @@ struct WgradArgs {
 };
 // Returns cudaSuccess or the failing CUDA error; *msg (static string) says which step failed.
 cudaError_t launch_wgrad_fold(const WgradArgs &args, const char **msg);
+// Several layers in ONE launch, worked through in the given order; stream, status block,
+// constants, variant and wait limit are taken from layers[0].  1 <= count <= kMaxWgradLayers.
+constexpr int kMaxWgradLayers = 8;
+cudaError_t launch_wgrad_fold_multi(const WgradArgs *layers, int count, const char **msg);
 // One-time, per process: resolves the driver's tensor-map encoder.
 cudaError_t wgrad_fold_setup(const char **msg);
 // Set-up bookkeeping, for diagnostics: bit 0 = the encoder has been resolved, bit 1 = the

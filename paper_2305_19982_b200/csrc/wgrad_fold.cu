@@ -379,8 +379,34 @@ __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars,
 // of the remaining full tiles: when the last round would occupy at most half of the CTA
 // groups, halving its tiles halves its duration (the token sum of each half is still
 // complete, so the square stays exact).
+//
+// One launch may cover several layers (adama_linear_wgrad_fold_multi): the work list is the
+// layers' lists one after the other, and a CTA pair walks through it with a stride of the
+// number of pairs.  The pairs that a layer's last round leaves idle therefore start on the
+// next layer, the epilogue of a layer's last tile overlaps the next layer's first main loop,
+// and set-up, pipeline fill and the one exposed epilogue are paid once per launch.
 struct WorkItem {
     int m0, n0, width;
+};
+// Everything the kernel needs to know about one layer (kernel parameter space).
+struct alignas(64) WgradLayer {
+    CUtensorMap map_x, map_dy;             // 2-D views, one 64-feature x 64-token box per operation
+    CUtensorMap map_x3, map_dy3, map_dy3h; // grouped 3-D views (d_in, d_out multiples of 64)
+    float *m, *v;
+    const __nv_bfloat16 *dy_raw;           // dY again, for the bias warps
+    float *bias_m, *bias_v;                // null: the layer has no bias moments to fold
+    long long ldmv, ldy;
+    int tokens, d_in, d_out, grouped;
+    int tiles_m, tiles_n;
+    int split_from;   // layer-local item index from which items are 128-column halves
+    int item_begin;   // index of the layer's first item in the launch's work list
+};
+constexpr int kMaxLayers = 8;
+struct WgradTable {
+    WgradLayer layer[kMaxLayers];
+    int count;       // layers in this launch
+    int num_items;   // work items of all layers
+    int any_bias;    // some layer has bias moments: the CTAs carry the two bias warps
 };
 __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m, int tiles_n) {
     int full = w, half = 0, width = BN;
@@ -394,19 +420,18 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
     const int tn = tiles_n < tiles_m ? full % tiles_n : full / tiles_m;
     return {tm * Geo<>::TILE_M, tn * BN + half * (BN / 2), width};
 }
+// The layer that item `w` of the launch belongs to, and the item within that layer.
+__device__ __forceinline__ const WgradLayer *layer_of(const WgradTable &tab, int w, WorkItem *wi) {
+    int l = 0;
+    while (l + 1 < tab.count && w >= tab.layer[l + 1].item_begin) ++l;
+    const WgradLayer *L = &tab.layer[l];
+    *wi = work_item(w - L->item_begin, L->split_from, L->tiles_m, L->tiles_n);
+    return L;
+}
 
 template <bool STAGED>
 __global__ void __launch_bounds__(STAGED ? STAGED_THREADS : MAX_THREADS, 1)
-wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
-                  const __grid_constant__ CUtensorMap map_dy,
-                  const __grid_constant__ CUtensorMap map_x3,
-                  const __grid_constant__ CUtensorMap map_dy3,
-                  const __grid_constant__ CUtensorMap map_dy3h, int grouped,
-                  float *__restrict__ m_out,
-                  float *__restrict__ v_out, long long ldmv, int tokens, int d_in, int d_out,
-                  int split_from, int num_items, float a, float b, unsigned *status,
-                  const __nv_bfloat16 *__restrict__ dy_raw, long long ldy,
-                  float *__restrict__ bias_m, float *__restrict__ bias_v,
+wgrad_fold_kernel(const __grid_constant__ WgradTable tab, float a, float b, unsigned *status,
                   unsigned long long wait_limit_ns, int withhold_last_load) {
     using G = Geo<STAGED>;
     constexpr int STAGES = G::STAGES;
@@ -422,13 +447,11 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
     const uint32_t rank = cluster_ctarank();  // position in the pair
     const int group = blockIdx.x / CTAS;                           // which pair
     const int num_groups = gridDim.x / CTAS;
-    const int tiles_m = (d_in + G::TILE_M - 1) / G::TILE_M;
-    const int tiles_n = (d_out + BN - 1) / BN;
-    const int num_kb = (tokens + BK - 1) / BK;
+    const int num_items = tab.num_items;
     // warps 2 .. 2+epi_warps-1: epilogue; with bias moments, BIAS_WARPS more after them
     // (staged: 4 drain warps take the epilogue's place, 8 streaming warps follow them)
     const int epi_warps = STAGED ? STAGED_DRAIN_WARPS
-                                 : (int)blockDim.x / 32 - 2 - (bias_m != nullptr ? BIAS_WARPS : 0);
+                                 : (int)blockDim.x / 32 - 2 - (tab.any_bias ? BIAS_WARPS : 0);
     const int first_bias_warp = 2 + epi_warps + (STAGED ? STAGED_STREAM_WARPS : 0);
 
     if (threadIdx.x == 0) {
@@ -474,7 +497,9 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             // the pair's loads are counted by the first CTA's barrier
             const uint32_t full0_lead = map_to_cta(full0, 0);
             for (int tile = group; tile < num_items && ok; tile += num_groups) {
-                const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
+                WorkItem wi;
+                const WgradLayer *L = layer_of(tab, tile, &wi);
+                const int num_kb = (L->tokens + BK - 1) / BK;
                 const int cols_per_cta = wi.width / CTAS;  // dY columns this CTA stages
                 const int b_boxes = cols_per_cta / GROUP;
                 const int m0 = wi.m0 + (int)rank * G::ROWS_PER_CTA;
@@ -495,18 +520,18 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     const uint32_t sb = sa + G::A_STAGE_BYTES;
                     // out-of-range parts of a box are zero-filled and still counted
                     if (rank == 0) mbar_arrive_expect_tx(full0 + (uint32_t)stage * 8u, stage_tx);
-                    if (grouped) {
+                    if (L->grouped) {
                         // d_in, d_out multiples of 64: one operation per operand
-                        tma_load_3d(sa, &map_x3, kb * BK, m0 / GROUP, bar);
-                        tma_load_3d(sb, b_boxes == G::B_BOXES ? &map_dy3 : &map_dy3h, kb * BK,
+                        tma_load_3d(sa, &L->map_x3, kb * BK, m0 / GROUP, bar);
+                        tma_load_3d(sb, b_boxes == G::B_BOXES ? &L->map_dy3 : &L->map_dy3h, kb * BK,
                                           n0 / GROUP, bar);
                     } else {
 #pragma unroll
                         for (int j = 0; j < G::A_BOXES; ++j)
-                            tma_load_2d(sa + j * BOX_BYTES, &map_x, m0 + j * GROUP, kb * BK,
+                            tma_load_2d(sa + j * BOX_BYTES, &L->map_x, m0 + j * GROUP, kb * BK,
                                               bar);
                         for (int j = 0; j < b_boxes; ++j)
-                            tma_load_2d(sb + j * BOX_BYTES, &map_dy, n0 + j * GROUP, kb * BK,
+                            tma_load_2d(sb + j * BOX_BYTES, &L->map_dy, n0 + j * GROUP, kb * BK,
                                               bar);
                     }
                     armed |= 1u << stage;
@@ -547,9 +572,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-                const uint32_t idesc =
-                    G::INSTR_DESC_NO_N |
-                    ((uint32_t)(work_item(tile, split_from, tiles_m, tiles_n).width >> 3) << 17);
+                WorkItem wi;
+                const WgradLayer *L = layer_of(tab, tile, &wi);
+                const int num_kb = (L->tokens + BK - 1) / BK;
+                const uint32_t idesc = G::INSTR_DESC_NO_N | ((uint32_t)(wi.width >> 3) << 17);
                 ok = mbar_wait(smem_u32(&bars->acc_empty[as]), aphase ^ 1, abort_flag, wait_limit_ns);
                 if (!ok) {
                     record_timeout(status, bars, 2, (unsigned)tile);
@@ -629,25 +655,30 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
 
         struct Part {
             float *pm, *pv;
-            int row_first, gcol;
+            long long ldmv;
+            int row_first, gcol, d_in, d_out;
             bool col_vec;
         };
         auto part_at = [&](int tile, int part_i) {
-            const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
+            WorkItem wi;
+            const WgradLayer *L = layer_of(tab, tile, &wi);
             Part u;
+            u.ldmv = L->ldmv;
+            u.d_in = L->d_in;
+            u.d_out = L->d_out;
             u.row_first = wi.m0 + (int)rank * G::ROWS_PER_CTA + lrow0;
             u.gcol = wi.n0 + part_i * PART_COLS + cl * 4;
-            u.col_vec = u.gcol + 4 <= d_out;  // whole group of four columns inside
-            u.pm = m_out + (long long)u.row_first * ldmv + u.gcol;
-            u.pv = v_out + (long long)u.row_first * ldmv + u.gcol;
+            u.col_vec = u.gcol + 4 <= u.d_out;  // whole group of four columns inside
+            u.pm = L->m + (long long)u.row_first * u.ldmv + u.gcol;
+            u.pv = L->v + (long long)u.row_first * u.ldmv + u.gcol;
             return u;
         };
         auto load_m = [&](const Part &u, float4(&mm)[8]) {
             if (u.col_vec) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                    if (u.row_first + i * RPI < d_in)
-                        mm[i] = ld_global_v4_stream(u.pm + (long long)(i * RPI) * ldmv);
+                    if (u.row_first + i * RPI < u.d_in)
+                        mm[i] = ld_global_v4_stream(u.pm + (long long)(i * RPI) * u.ldmv);
             }
         };
         // waits for part buffer k to hold the part, folds it, hands the buffer back
@@ -663,7 +694,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             if (u.col_vec) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                    if (u.row_first + i * RPI < d_in) {
+                    if (u.row_first + i * RPI < u.d_in) {
                         const int lrow = lrow0 + i * RPI;
                         const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
                                                       (uint32_t)((cl ^ (lrow & 7)) << 4));
@@ -672,25 +703,25 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                         x.y = fmaf(a, g.y, x.y);
                         x.z = fmaf(a, g.z, x.z);
                         x.w = fmaf(a, g.w, x.w);
-                        st_global_v4(u.pm + (long long)(i * RPI) * ldmv, x);
-                        red_add_v4(u.pv + (long long)(i * RPI) * ldmv,
+                        st_global_v4(u.pm + (long long)(i * RPI) * u.ldmv, x);
+                        red_add_v4(u.pv + (long long)(i * RPI) * u.ldmv,
                                    make_float4((b * g.x) * g.x, (b * g.y) * g.y, (b * g.z) * g.z,
                                                (b * g.w) * g.w));
                     }
-            } else if (u.gcol < d_out) {
+            } else if (u.gcol < u.d_out) {
                 // last, partial group of four columns: element-wise
                 for (int i = 0; i < 8; ++i) {
                     const int lrow = lrow0 + i * RPI;
-                    if (u.row_first + i * RPI >= d_in) break;
+                    if (u.row_first + i * RPI >= u.d_in) break;
                     const float4 g = ld_shared_v4(pbuf + (uint32_t)lrow * PITCH +
                                                   (uint32_t)((cl ^ (lrow & 7)) << 4));
                     const float ge[4] = {g.x, g.y, g.z, g.w};
                     for (int e = 0; e < 4; ++e)
-                        if (u.gcol + e < d_out) {
-                            float *qm = u.pm + (long long)(i * RPI) * ldmv + e;
-                            float *qv = u.pv + (long long)(i * RPI) * ldmv + e;
+                        if (u.gcol + e < u.d_out) {
+                            float *qm = u.pm + (long long)(i * RPI) * u.ldmv + e;
+                            float *qv = u.pv + (long long)(i * RPI) * u.ldmv + e;
                             *qm = fmaf(a, ge[e], *qm);
-                            *qv += (b * ge[e]) * ge[e];
+                            *qv = __fadd_rn(*qv, __fmul_rn(__fmul_rn(b, ge[e]), ge[e]));  // as the reduction rounds
                         }
                 }
             }
@@ -704,7 +735,9 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             load_m(u_a, m_a);
             for (int tile = group; tile < num_items && ok; tile += num_groups) {
                 // parts per tile: 4 (full tile) or 2 (half tile); part i lives in buffer i & 1
-                const int nparts = work_item(tile, split_from, tiles_m, tiles_n).width / PART_COLS;
+                WorkItem wi_t;
+                layer_of(tab, tile, &wi_t);
+                const int nparts = wi_t.width / PART_COLS;
                 for (int part_i = 0; part_i < nparts && ok; part_i += 2) {
                     u_b = part_at(tile, part_i + 1);
                     load_m(u_b, m_b);
@@ -734,11 +767,18 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         // between them cannot be left waiting by a role that gave up.
         grid_dependency_wait();
         const int ew = warp - first_bias_warp;
-        const int slabs = (d_out + 31) / 32;
         float *red = reinterpret_cast<float *>(smem + G::SMEM_BIAS_OFF);  // [BIAS_WARPS][32]
         const int rsub = lane >> 2;  // row within a group of 8
         const int cq = lane & 3;     // 16-byte chunk of the slab's 64-byte row segment
         const int step = BIAS_WARPS * 8;
+        for (int l = 0; l < tab.count; ++l) {
+        const WgradLayer *L = &tab.layer[l];
+        float *bias_m = L->bias_m, *bias_v = L->bias_v;
+        if (bias_m == nullptr) continue;  // (uniform over the two warps)
+        const int d_out = L->d_out, tokens = L->tokens;
+        const long long ldy = L->ldy;
+        const __nv_bfloat16 *dy_raw = L->dy_raw;
+        const int slabs = (d_out + 31) / 32;
         for (int slab = (int)blockIdx.x; slab < slabs; slab += (int)gridDim.x) {
             const int col = slab * 32 + cq * 8;
             float acc[8];
@@ -801,6 +841,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             }
             asm volatile("bar.sync 1, %0;" ::"r"(BIAS_WARPS * 32) : "memory");
         }
+        }  // layers
     } else {
         if constexpr (STAGED) {
             // ---------------- staged epilogue, drain side: accumulator -> shared-memory tile ----------------
@@ -815,7 +856,8 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-                const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
+                WorkItem wi;
+                layer_of(tab, tile, &wi);
                 ok = mbar_wait(smem_u32(&bars->acc_full[as]), aphase, abort_flag, wait_limit_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) {
@@ -889,6 +931,10 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
             int col0;
             bool inside, interior;
         };
+        // the layer of the tile at hand (set per tile; the helpers below read it)
+        float *m_out = nullptr, *v_out = nullptr;
+        long long ldmv = 0;
+        int d_in = 0, d_out = 0;
         auto chunk_at = [&](const WorkItem &wi, int row0, int c) {
             Chunk ch;
             ch.col0 = wi.n0 + c * EPI_COLS;
@@ -944,7 +990,7 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
                     for (int e = 0; e < 4; ++e)
                         if (ch.col0 + c4 * 4 + e < d_out) {
                             pm[e] = fmaf(a, ge[e], pm[e]);
-                            pv[e] += (b * ge[e]) * ge[e];
+                            pv[e] = __fadd_rn(pv[e], __fmul_rn(__fmul_rn(b, ge[e]), ge[e]));  // as the reduction rounds
                         }
                 }
             }
@@ -953,7 +999,13 @@ wgrad_fold_kernel(const __grid_constant__ CUtensorMap map_x,
         for (int tile = group; tile < num_items && ok; tile += num_groups, ++it) {
             const int as = it & 1;
             const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
-            const WorkItem wi = work_item(tile, split_from, tiles_m, tiles_n);
+            WorkItem wi;
+            const WgradLayer *L = layer_of(tab, tile, &wi);
+            m_out = L->m;
+            v_out = L->v;
+            ldmv = L->ldmv;
+            d_in = L->d_in;
+            d_out = L->d_out;
             const int row0 = wi.m0 + (int)rank * G::ROWS_PER_CTA + q * EPI_ROWS;
             const int chunks = wi.width / (col_split * EPI_COLS);  // chunks per warp
             const int c_first = part * chunks;
@@ -1097,50 +1149,85 @@ static cudaError_t ensure_device_attributes(const char **msg) {
     return cudaSuccess;
 }
 
-cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
-    cudaError_t e = wgrad_fold_setup(msg);
-    if (e == cudaSuccess) e = ensure_device_attributes(msg);
-    if (e != cudaSuccess) return e;
-    CUtensorMap map_x, map_dy;
-    bool ok = encode_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.X, (uint64_t)p.d_in,
+// Fills one layer's entry of the kernel's table; *tiles = the layer's full 256x256 tiles.
+static bool fill_layer(const WgradArgs &p, WgradLayer *L, int *tiles) {
+    bool ok = encode_2d(&L->map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.X, (uint64_t)p.d_in,
                         (uint64_t)p.tokens, (uint64_t)p.ldx, GROUP, BK,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B) &&
-              encode_2d(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.dY, (uint64_t)p.d_out,
+              encode_2d(&L->map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.dY, (uint64_t)p.d_out,
                         (uint64_t)p.tokens, (uint64_t)p.ldy, GROUP, BK,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     // grouped loads need whole 64-feature groups in both operands
-    CUtensorMap map_x3 = map_x, map_dy3 = map_dy, map_dy3h = map_dy;
-    int grouped = (p.d_in % GROUP == 0 && p.d_out % GROUP == 0 && !p.variant.box_loads) ? 1 : 0;
-    if (ok && grouped)
-        ok = encode_grouped(&map_x3, p.X, (uint64_t)p.d_in, (uint64_t)p.tokens, (uint64_t)p.ldx, BK,
-                            Geo<>::A_BOXES) &&
-             encode_grouped(&map_dy3, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens, (uint64_t)p.ldy,
-                            BK, Geo<>::B_BOXES) &&
-             encode_grouped(&map_dy3h, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens,
+    L->map_x3 = L->map_x;
+    L->map_dy3 = L->map_dy;
+    L->map_dy3h = L->map_dy;
+    L->grouped = (p.d_in % GROUP == 0 && p.d_out % GROUP == 0 && !p.variant.box_loads) ? 1 : 0;
+    if (ok && L->grouped)
+        ok = encode_grouped(&L->map_x3, p.X, (uint64_t)p.d_in, (uint64_t)p.tokens, (uint64_t)p.ldx,
+                            BK, Geo<>::A_BOXES) &&
+             encode_grouped(&L->map_dy3, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens,
+                            (uint64_t)p.ldy, BK, Geo<>::B_BOXES) &&
+             encode_grouped(&L->map_dy3h, p.dY, (uint64_t)p.d_out, (uint64_t)p.tokens,
                             (uint64_t)p.ldy, BK, Geo<>::B_BOXES / 2);
-    if (!ok) {
-        *msg = "cuTensorMapEncodeTiled rejected a tensor";
+    L->m = p.m;
+    L->v = p.v;
+    L->dy_raw = static_cast<const __nv_bfloat16 *>(p.dY);
+    L->bias_m = p.bias_m;
+    L->bias_v = p.bias_v;
+    L->ldmv = (long long)p.ldmv;
+    L->ldy = (long long)p.ldy;
+    L->tokens = p.tokens;
+    L->d_in = p.d_in;
+    L->d_out = p.d_out;
+    L->tiles_m = (p.d_in + Geo<>::TILE_M - 1) / Geo<>::TILE_M;
+    L->tiles_n = (p.d_out + BN - 1) / BN;
+    *tiles = L->tiles_m * L->tiles_n;
+    L->split_from = *tiles;  // no halves unless the launch's tail says so
+    return ok;
+}
+
+cudaError_t launch_wgrad_fold_multi(const WgradArgs *layers, int count, const char **msg) {
+    if (count < 1 || count > kMaxWgradLayers) {
+        *msg = "wgrad_fold: layer count out of range";
         return cudaErrorInvalidValue;
     }
-    const int tiles_n = (p.d_out + BN - 1) / BN;
-    *msg = "wgrad_fold launch";
-    const int tiles = ((p.d_in + Geo<>::TILE_M - 1) / Geo<>::TILE_M) * tiles_n;
-    const int max_groups = p.sm_count / 2;
-    // Tail balancing: if the last round would keep at most half of the groups busy, its
-    // tiles are issued as 128-column halves (see WorkItem).
-    const int rest = tiles % max_groups;
-    int split_from = tiles, items = tiles;
-    if (rest > 0 && 2 * rest <= max_groups) {
-        split_from = tiles - rest;
-        items = tiles + rest;
+    cudaError_t e = wgrad_fold_setup(msg);
+    if (e == cudaSuccess) e = ensure_device_attributes(msg);
+    if (e != cudaSuccess) return e;
+    const WgradArgs &p = layers[0];  // stream, status block, constants, variant: the launch's
+    static_assert(kMaxWgradLayers == kMaxLayers, "table size");
+    WgradTable tab = {};
+    tab.count = count;
+    int items = 0, max_tokens = 0, min_tokens = layers[0].tokens;
+    int tiles_of[kMaxLayers];
+    for (int l = 0; l < count; ++l) {
+        if (!fill_layer(layers[l], &tab.layer[l], &tiles_of[l])) {
+            *msg = "cuTensorMapEncodeTiled rejected a tensor";
+            return cudaErrorInvalidValue;
+        }
+        tab.layer[l].item_begin = items;
+        items += tiles_of[l];
+        if (layers[l].bias_m) tab.any_bias = 1;
+        max_tokens = layers[l].tokens > max_tokens ? layers[l].tokens : max_tokens;
+        min_tokens = layers[l].tokens < min_tokens ? layers[l].tokens : min_tokens;
     }
+    *msg = "wgrad_fold launch";
+    const int max_groups = p.sm_count / 2;
+    // Tail balancing: if the launch's last round would keep at most half of the groups busy, its
+    // tiles (the last layer's last ones) are issued as 128-column halves (see WorkItem).
+    const int rest = items % max_groups;
+    if (rest > 0 && 2 * rest <= max_groups && rest <= tiles_of[count - 1]) {
+        tab.layer[count - 1].split_from = tiles_of[count - 1] - rest;
+        items += rest;
+    }
+    tab.num_items = items;
     const int groups = items < max_groups ? items : max_groups;
     // 8 epilogue warps when no CTA group gets a second tile (exposed epilogue) or when the
     // contraction is short (up to 2048 tokens the m, v traffic of the epilogue, not the tensor
     // cores, bounds the call: 4096x4096 with 1024 tokens 78.9 vs 82.9 us), else 4
     const bool wide = p.variant.epi_warps ? p.variant.epi_warps == 8
-                                          : (items <= max_groups || p.tokens <= 2048);
-    const int threads = 32 * (2 + (wide ? MAX_EPI_WARPS : 4) + (p.bias_m ? BIAS_WARPS : 0));
+                                          : (items <= max_groups || max_tokens <= 2048);
+    const int threads = 32 * (2 + (wide ? MAX_EPI_WARPS : 4) + (tab.any_bias ? BIAS_WARPS : 0));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * groups), 1, 1);
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
@@ -1148,9 +1235,9 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     // (4096x4096, L2 flushed, staged vs direct epilogue, us: 256 tokens 65.6 vs 75.8, 1024: 69.7 vs
     // 79.9, 2048: 75.8 vs 82.0, 3072: 94.2 vs 92.2, 4096: 114.7 vs 110.6.  With 128-column parts and
     // the 3-stage ring they leave: 66.6, 71.7, 92.2 at 256, 1024, 2048 tokens.)
-    const bool staged = p.variant.epilogue ? p.variant.epilogue == 2 : p.tokens <= 2048;
+    const bool staged = p.variant.epilogue ? p.variant.epilogue == 2 : max_tokens <= 2048;
     cfg.dynamicSmemBytes = staged ? Geo<true>::SMEM_BYTES : Geo<>::SMEM_BYTES;
-    if (staged) cfg.blockDim = dim3((unsigned)(STAGED_THREADS - (p.bias_m ? 0 : 32 * BIAS_WARPS)), 1, 1);
+    if (staged) cfg.blockDim = dim3((unsigned)(STAGED_THREADS - (tab.any_bias ? 0 : 32 * BIAS_WARPS)), 1, 1);
     cfg.stream = p.stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1163,11 +1250,12 @@ cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
     cfg.attrs = attr;
     cfg.numAttrs = p.variant.no_pdl ? 1 : 2;
     const unsigned long long limit = p.wait_limit_ns ? p.wait_limit_ns : kDefaultWaitLimitNs;
-    return cudaLaunchKernelEx(&cfg, staged ? wgrad_fold_kernel<true> : wgrad_fold_kernel<false>,
-                              map_x, map_dy, map_x3, map_dy3, map_dy3h, grouped, p.m, p.v,
-                              (long long)p.ldmv, p.tokens, p.d_in, p.d_out, split_from, items,
-                              p.c.a, p.c.b, p.status, static_cast<const __nv_bfloat16 *>(p.dY),
-                              (long long)p.ldy, p.bias_m, p.bias_v, limit, p.withhold_last_load);
+    return cudaLaunchKernelEx(&cfg, staged ? wgrad_fold_kernel<true> : wgrad_fold_kernel<false>, tab,
+                              p.c.a, p.c.b, p.status, limit, p.withhold_last_load);
+}
+
+cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {
+    return launch_wgrad_fold_multi(&p, 1, msg);
 }
 
 }  // namespace adama

@@ -63,22 +63,37 @@ class LinearStack:
         return sum(2.0 * tokens * L.d_in * L.d_out for L in self.layers)
 
     def fold_micro_batches(self, opt: AdamA, n_micro: int,
-                           inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]]) -> None:
+                           inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]],
+                           layers_per_launch: int = 1) -> None:
         """The accumulation half of one mini-batch (Algorithm 2, inner loops): begin, then for
         every micro-batch every layer from the last to the first through the fused
         weight-gradient fold.  `inputs(micro, layer_index, spec)` returns (X, dY) for that
-        (micro-batch, layer); the tensors are released right after the layer's call.  The
-        weight gradient never exists in memory.  On return m, v hold m_t, v_t."""
+        (micro-batch, layer).  The weight gradient never exists in memory.  On return m, v
+        hold m_t, v_t.
+
+        layers_per_launch = 1: one call per layer, its (X, dY) released right after the call.
+        layers_per_launch = k > 1: k consecutive layers (still back to front) go into one
+        adama_linear_wgrad_fold_multi call, e.g. the four linears of a transformer block; their
+        (X, dY) are released together after that call.  Same results, bit for bit."""
         opt.begin_minibatch(n_micro)
         for i in range(n_micro):
+            pending = []
             for j in reversed(range(len(self.layers))):
                 X, dY = inputs(i, j, self.layers[j])
+                item = (X, dY, self.view(self.m, j), self.view(self.v, j))
                 if self.biases:  # bias gradient (column sums of dY) in the same launch
-                    opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j),
-                                          self.bias_view(self.m, j), self.bias_view(self.v, j))
-                else:
-                    opt.linear_wgrad_fold(X, dY, self.view(self.m, j), self.view(self.v, j))
+                    item += (self.bias_view(self.m, j), self.bias_view(self.v, j))
                 del X, dY
+                if layers_per_launch <= 1:
+                    opt.linear_wgrad_fold(*item)
+                else:
+                    pending.append(item)
+                    if len(pending) == layers_per_launch:
+                        opt.linear_wgrad_fold_multi(pending)
+                        pending = []
+                del item
+            if pending:
+                opt.linear_wgrad_fold_multi(pending)
 
     def apply(self, opt: AdamA, lr: float) -> None:
         """The update half (Algorithm 2, "Update"): one apply over the whole flat buffer (the
@@ -86,9 +101,10 @@ class LinearStack:
         opt.apply(self.w, self.m, self.v, lr)
 
     def minibatch(self, opt: AdamA, n_micro: int, lr: float,
-                  inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]]) -> None:
+                  inputs: Callable[[int, int, LayerSpec], Tuple[torch.Tensor, torch.Tensor]],
+                  layers_per_launch: int = 1) -> None:
         """One whole mini-batch: fold_micro_batches, then apply."""
-        self.fold_micro_batches(opt, n_micro, inputs)
+        self.fold_micro_batches(opt, n_micro, inputs, layers_per_launch)
         self.apply(opt, lr)
 
 

@@ -18,8 +18,8 @@ pytestmark = pytest.mark.gpu
 TOL_BF16 = 2e-3
 
 
-@pytest.mark.parametrize("biases", [False, True])
-def test_small_stack_full_parity(biases):
+@pytest.mark.parametrize("biases,per_launch", [(False, 1), (True, 1), (False, 2), (True, 3)])
+def test_small_stack_full_parity(biases, per_launch):
     layers = [LayerSpec("a", 200, 328), LayerSpec("b", 328, 136), LayerSpec("c", 136, 8)]
     T, N, steps = 192, 2, 2
     stack = LinearStack(layers, biases=biases)
@@ -41,7 +41,7 @@ def test_small_stack_full_parity(biases):
             if biases:      # bias gradient = column sums of dY (naive loop in the oracle)
                 borcs[j].fold(oracle.linear_wgrad(np.ones((T, 1)), f64(dY))[0])
             return X.cuda(), dY.cuda()
-        stack.fold_micro_batches(opt, N, inputs)
+        stack.fold_micro_batches(opt, N, inputs, layers_per_launch=per_launch)
         opt.sync_status()
         for j in range(len(layers)):   # m_t, v_t after the last fold of the mini-batch
             assert_close(f64(stack.view(stack.m, j)), orcs[j].m, TOL_BF16, f"m_t layer {j}")
@@ -64,7 +64,7 @@ def test_small_stack_full_parity(biases):
 
 
 def _sampled_stack(stack: LinearStack, tokens: int, n_micro: int, steps: int, config: int,
-                   per_layer: int):
+                   per_layer: int, layers_per_launch: int = 1):
     """`steps` mini-batches of `n_micro` micro-batches over every layer of the stack, in the
     launch configuration the benchmark times.  Per layer a fixed sample of entries (random ones
     plus the first and the last row / column) is followed through the whole recurrence by the
@@ -98,7 +98,7 @@ def _sampled_stack(stack: LinearStack, tokens: int, n_micro: int, steps: int, co
             orc.fold(G, lo=j * S)
             return X, dY
 
-        stack.fold_micro_batches(opt, n_micro, inputs)
+        stack.fold_micro_batches(opt, n_micro, inputs, layers_per_launch)
         opt.sync_status()
         assert_close(f64(stack.m[flat]), orc.m, TOL_BF16, f"m_t step {step}")
         assert_close(f64(stack.v[flat]), orc.v, TOL_BF16, f"v_t step {step}")
@@ -120,6 +120,13 @@ def test_gpt2xl_full_stack_sampled():
     stack = gpt2xl_stack(wl.CONFIG4_BLOCKS)
     assert stack.n_params == 48 * (1600 * 4800 + 1600 * 1600 + 2 * 1600 * 6400)
     _sampled_stack(stack, wl.CONFIG4_TOKENS, wl.CONFIG4_N_MICRO, 2, 4, 24)
+
+
+def test_gpt2xl_full_stack_one_launch_per_block_sampled():
+    """The same stack with the four linears of a block folded by one grouped launch
+    (adama_linear_wgrad_fold_multi), N = 8, 2 mini-batches."""
+    stack = gpt2xl_stack(wl.CONFIG4_BLOCKS)
+    _sampled_stack(stack, wl.CONFIG4_TOKENS, wl.CONFIG4_N_MICRO, 2, 4, 24, layers_per_launch=4)
 
 
 def test_llama7b_two_blocks_sampled():

@@ -178,6 +178,74 @@ def test_variant_entry_rejects_values_out_of_range():
     opt.close()
 
 
+def test_multi_layer_launch_equals_per_layer_calls_and_the_oracle():
+    """adama_linear_wgrad_fold_multi: ten layers of assorted shapes (ragged, more tiles than CTA
+    pairs, a single tile, token counts on both sides of the short-call limit, two with bias
+    moments) in one call -- two launches, since a launch takes at most eight.  Every layer must
+    come out bit for bit as from its own adama_linear_wgrad_fold / _bias_fold call, and (integer
+    inputs: exact contraction) match the oracle at the fp32 fold tolerance, element by element."""
+    specs = [(192, 200, 328, False), (320, 512, 768, True), (64, 136, 8, False), (192, 2560, 2048, False),
+             (2240, 304, 1000, False), (100, 128, 256, True), (640, 1600, 1600, False), (7, 136, 264, False),
+             (256, 768, 512, False), (2112, 640, 1280, False)]
+    N = 3
+    single, multi = adama.AdamA(), adama.AdamA()
+    single.begin_minibatch(N)
+    multi.begin_minibatch(N)
+    layers_s, layers_m, orcs, borcs = [], [], [], []
+    for k, (T, d_in, d_out, bias) in enumerate(specs):
+        z = lambda *shape: torch.zeros(*shape, device="cuda")
+        layers_s.append([z(d_in, d_out), z(d_in, d_out)] + ([z(d_out), z(d_out)] if bias else []))
+        layers_m.append([z(d_in, d_out), z(d_in, d_out)] + ([z(d_out), z(d_out)] if bias else []))
+        o = AdamAOracle(np.zeros((d_in, d_out)))
+        o.begin_minibatch(N)
+        orcs.append(o)
+        bo = AdamAOracle(np.zeros(d_out))
+        bo.begin_minibatch(N)
+        borcs.append(bo)
+    for i in range(N):
+        items = []
+        for k, (T, d_in, d_out, bias) in enumerate(specs):
+            X, dY = _draw(T, d_in, d_out, 5000 + 100 * i + k, integer=True)
+            orcs[k].fold_linear(f64(X), f64(dY))
+            if bias:
+                borcs[k].fold(oracle.linear_wgrad(np.ones((T, 1)), f64(dY))[0])
+            X, dY = X.cuda(), dY.cuda()
+            single.linear_wgrad_fold(X, dY, *layers_s[k])
+            items.append((X, dY, *layers_m[k]))
+        before = multi.launch_count
+        multi.linear_wgrad_fold_multi(items)
+        assert multi.launch_count - before == 2
+    single.sync_status()
+    multi.sync_status()
+    for k, (T, d_in, d_out, bias) in enumerate(specs):
+        for a, b in zip(layers_s[k], layers_m[k]):
+            assert torch.equal(a, b), f"layer {k}: grouped launch differs from the per-layer call"
+        assert_close(f64(layers_m[k][0]), orcs[k].m, TOL_EXACT, f"m layer {k}")
+        assert_close(f64(layers_m[k][1]), orcs[k].v, TOL_EXACT, f"v layer {k}")
+        if bias:
+            assert_close(f64(layers_m[k][2]), borcs[k].m, TOL_EXACT, f"bias m layer {k}")
+            assert_close(f64(layers_m[k][3]), borcs[k].v, TOL_EXACT, f"bias v layer {k}")
+    single.close()
+    multi.close()
+
+
+def test_multi_layer_call_checks_every_item_before_launching():
+    opt = adama.AdamA()
+    opt.begin_minibatch(1)
+    X = torch.zeros(64, 128, dtype=torch.bfloat16, device="cuda")
+    dY = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
+    m = torch.zeros(128, 256, device="cuda")
+    bad = torch.zeros(64 * 128 + 8, dtype=torch.bfloat16, device="cuda")[1:1 + 64 * 128].view(64, 128)
+    with pytest.raises(adama.AdamAError) as e:
+        opt.linear_wgrad_fold_multi([(X, dY, m, m.clone()), (bad, dY, m.clone(), m.clone())])
+    assert e.value.status == adama.Status.ERR_MISALIGNED and opt.launch_count == 0
+    opt.linear_wgrad_fold_multi([])                      # nothing to do
+    e0 = torch.empty(0, 128, dtype=torch.bfloat16, device="cuda")
+    opt.linear_wgrad_fold_multi([(e0, torch.empty(0, 256, dtype=torch.bfloat16, device="cuda"), m, m.clone())])
+    assert opt.launch_count == 0                         # zero tokens: skipped
+    opt.close()
+
+
 def test_long_contraction_phase_wraps():
     _full_parity(4096 + 48, 256, 512, n_micro=1)
 
