@@ -915,6 +915,27 @@ def run_wgrad_shapes(args):
         ts.sort()
         return ts[len(ts) // 2]
 
+    def timed_in_model(d_in, d_out, make_call, reps=3):
+        # as inside a model: calls back to back, each on its own copy of the layer's m and v, enough
+        # copies that a call never finds its states in the L2 (>= 640 MB of states in the cycle);
+        # no launch bubble as around a single call, no warm L2 as with one buffer
+        copies = max(2, -(-(640 << 20) // (8 * d_in * d_out)))
+        states = [(torch.zeros(d_in, d_out, device=dev), torch.zeros(d_in, d_out, device=dev))
+                  for _ in range(copies)]
+        for mm, vv in states:
+            make_call(mm, vv)
+        torch.cuda.synchronize()
+        time.sleep(0.5)
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for mm, vv in states:
+                make_call(mm, vv)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * copies) * 1e3
+
     rows = []
     for d_in, d_out in shapes:
         X = wl.normal((T, d_in), 1.0, torch.bfloat16, 1, device=dev)
@@ -943,7 +964,12 @@ def run_wgrad_shapes(args):
         cold_sep = rested(timed_cold, both)
         tf = 2.0 * T * d_in * d_out / us / 1e6
         tf_cold = 2.0 * T * d_in * d_out / cold / 1e6
+        us_model = timed_in_model(d_in, d_out, lambda mm, vv: opt.linear_wgrad_fold(X, dY, mm, vv))
+        tf_model = 2.0 * T * d_in * d_out / us_model / 1e6
         rows.append({"d_in": d_in, "d_out": d_out, "tokens": T,
+                     "in_model": {"us": us_model, "TFLOPps": tf_model,
+                                  "frac_of_burst_peak": tf_model / pk["bf16_tflops"],
+                                  "frac_of_sustained_peak": tf_model / pk["bf16_tflops_sustained"]},
                      "back_to_back": {"us": us, "TFLOPps": tf,
                                       "frac_of_burst_peak": tf / pk["bf16_tflops"],
                                       "us_with_fused_bias": us_fused,
@@ -965,17 +991,63 @@ def run_wgrad_shapes(args):
         torch.cuda.synchronize()
         time.sleep(0.5)
         us = timed_cold(lambda: opt.linear_wgrad_fold(X, dY, m, v))
+        us_model = timed_in_model(d_in, d_out, lambda mm, vv: opt.linear_wgrad_fold(X, dY, mm, vv))
         byts = 16 * d_in * d_out + 2 * tokens * (d_in + d_out)
         sweep.append({"tokens": tokens, "us": us, "TFLOPps": 2.0 * tokens * d_in * d_out / us / 1e6,
                       "hbm_GBps": byts / us / 1e3,
+                      "in_model_us": us_model, "in_model_hbm_GBps": byts / us_model / 1e3,
+                      "in_model_frac_of_hbm_peak": byts / us_model / 1e3 / pk["hbm_gbs"],
+                      "in_model_TFLOPps": 2.0 * tokens * d_in * d_out / us_model / 1e6,
                       "hbm_floor_us": byts / pk["hbm_gbs"] / 1e3,
                       "tensor_floor_us": 2.0 * tokens * d_in * d_out / pk["bf16_tflops"] / 1e6})
         del X, dY
+    # the linears of one transformer block folded by ONE grouped launch (adama_linear_wgrad_fold_multi),
+    # back to front, timed like "in_model" over enough copies of the block's states
+    blocks = []
+    for name, linears in (("gpt2xl_block", list(wl.gpt2xl_block_linears())),
+                          ("llama7b_block", list(wl.llama7b_block_linears()))):
+        linears = linears[::-1]
+        state_bytes = sum(8 * di * do for _, di, do in linears)
+        copies = max(2, -(-(640 << 20) // state_bytes))
+        xs = {d: wl.normal((T, d), 1.0, torch.bfloat16, 5 + d, device=dev) for d in {di for _, di, _ in linears}}
+        ys = {d: wl.normal((T, d), 1e-2, torch.bfloat16, 6 + d, device=dev) for d in {do for _, _, do in linears}}
+        groups = [[(xs[di], ys[do], torch.zeros(di, do, device=dev), torch.zeros(di, do, device=dev))
+                   for _, di, do in linears] for _ in range(copies)]
+        res = {}
+        for mode in ("one_launch_per_block", "one_launch_per_layer"):
+            def run(g):
+                if mode == "one_launch_per_block":
+                    opt.linear_wgrad_fold_multi(g)
+                else:
+                    for item in g:
+                        opt.linear_wgrad_fold(*item)
+            for g in groups:
+                run(g)
+            torch.cuda.synchronize()
+            time.sleep(0.5)
+            reps = 3
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                for g in groups:
+                    run(g)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / (reps * copies) * 1e3
+            tf = sum(2.0 * T * di * do for _, di, do in linears) / us / 1e6
+            res[mode] = {"us_per_block": us, "TFLOPps": tf, "frac_of_burst_peak": tf / pk["bf16_tflops"],
+                         "frac_of_sustained_peak": tf / pk["bf16_tflops_sustained"]}
+        blocks.append({"block": name, "layers": [[di, do] for _, di, do in linears], "tokens": T, **res})
+        del groups, xs, ys
     opt.sync_status()
-    print(json.dumps({"metric": "adama_wgrad_fold_per_shape", "token_sweep_4096x4096_l2_flushed": sweep, "unit": "us", "peak_tflops": pk["bf16_tflops"],
+    print(json.dumps({"metric": "adama_wgrad_fold_per_shape", "token_sweep_4096x4096_l2_flushed": sweep,
+                      "blocks_in_model": blocks, "unit": "us", "peak_tflops": pk["bf16_tflops"],
                       "peak_source": pk["source"],
                       "timing": "back_to_back: 20 calls between two CUDA events (buffers may stay in "
-                                "the L2); l2_flushed: median of 10 single calls, 512 MB written before each",
+                                "the L2); l2_flushed: median of 10 single calls, 512 MB written before each; "
+                                "in_model: calls back to back, each on its own copy of m and v, >= 640 MB of "
+                                "states in the cycle (cold L2, no single-call launch bubble)",
                       "rows": rows}), flush=True)
     opt.close()
 

@@ -179,14 +179,20 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
+// One probe of a barrier phase.  The explicit suspend-time hint matters: with it a thread that
+// waits on a barrier is back ~250 clocks sooner after the phase completes than with the default
+// time limit, and both the producer (waiting for a free stage) and the MMA issuer (waiting for a
+// full one) sit on the critical path of the operand ring (config-3 call 120.9 -> 118.8 us,
+// 4096x11008 305 -> 300 us; any hint from 32 ns to 2 us measured the same).
+constexpr uint32_t kSuspendHintNs = 64;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }
@@ -375,6 +381,10 @@ __device__ __forceinline__ void record_timeout(unsigned *status, Barriers *bars,
 // time then span a nearly square block of the tile grid and share the fewest distinct operand
 // blocks in the L2 (11008 x 4096 is 43 x 16 tiles: 74 consecutive tiles touch 5 row blocks and
 // 16 column blocks with the column index fastest, 43 and 2 with the row index fastest).
+// Calls of few tokens (the staged instance) are bound by the m, v traffic instead, and number
+// the tiles with the column index fastest whatever the shape: the tiles in flight then cover
+// whole rows of m and v (4096 x 4096, 2048 tokens: 74.0 us against 81.5; 1024 tokens: 62.9
+// against 67.7; 4096 x 11008, 1024 tokens: 146.5 against 162.4).
 // Items from split_from on are the two 128-column halves
 // of the remaining full tiles: when the last round would occupy at most half of the CTA
 // groups, halving its tiles halves its duration (the token sum of each half is still
@@ -400,6 +410,7 @@ struct alignas(64) WgradLayer {
     int tiles_m, tiles_n;
     int split_from;   // layer-local item index from which items are 128-column halves
     int item_begin;   // index of the layer's first item in the launch's work list
+    int col_fastest;  // tile numbering: column index fastest (else the row index)
 };
 constexpr int kMaxLayers = 8;
 struct WgradTable {
@@ -408,7 +419,8 @@ struct WgradTable {
     int num_items;   // work items of all layers
     int any_bias;    // some layer has bias moments: the CTAs carry the two bias warps
 };
-__device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m, int tiles_n) {
+__device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m, int tiles_n,
+                                              int col_fastest) {
     int full = w, half = 0, width = BN;
     if (w >= split_from) {
         const int j = w - split_from;
@@ -416,8 +428,8 @@ __device__ __forceinline__ WorkItem work_item(int w, int split_from, int tiles_m
         half = j & 1;
         width = BN / 2;
     }
-    const int tm = tiles_n < tiles_m ? full / tiles_n : full % tiles_m;
-    const int tn = tiles_n < tiles_m ? full % tiles_n : full / tiles_m;
+    const int tm = col_fastest ? full / tiles_n : full % tiles_m;
+    const int tn = col_fastest ? full % tiles_n : full / tiles_m;
     return {tm * Geo<>::TILE_M, tn * BN + half * (BN / 2), width};
 }
 // The layer that item `w` of the launch belongs to, and the item within that layer.
@@ -425,7 +437,7 @@ __device__ __forceinline__ const WgradLayer *layer_of(const WgradTable &tab, int
     int l = 0;
     while (l + 1 < tab.count && w >= tab.layer[l + 1].item_begin) ++l;
     const WgradLayer *L = &tab.layer[l];
-    *wi = work_item(w - L->item_begin, L->split_from, L->tiles_m, L->tiles_n);
+    *wi = work_item(w - L->item_begin, L->split_from, L->tiles_m, L->tiles_n, L->col_fastest);
     return L;
 }
 
@@ -1183,6 +1195,7 @@ static bool fill_layer(const WgradArgs &p, WgradLayer *L, int *tiles) {
     L->tiles_n = (p.d_out + BN - 1) / BN;
     *tiles = L->tiles_m * L->tiles_n;
     L->split_from = *tiles;  // no halves unless the launch's tail says so
+    L->col_fastest = L->tiles_n < L->tiles_m ? 1 : 0;  // shorter dimension fastest (see WorkItem)
     return ok;
 }
 
@@ -1237,6 +1250,8 @@ cudaError_t launch_wgrad_fold_multi(const WgradArgs *layers, int count, const ch
     // the 3-stage ring they leave: 66.6, 71.7, 92.2 at 256, 1024, 2048 tokens.)
     const bool staged = p.variant.epilogue ? p.variant.epilogue == 2 : max_tokens <= 2048;
     cfg.dynamicSmemBytes = staged ? Geo<true>::SMEM_BYTES : Geo<>::SMEM_BYTES;
+    if (staged)
+        for (int l = 0; l < count; ++l) tab.layer[l].col_fastest = 1;  // whole rows of m, v in flight
     if (staged) cfg.blockDim = dim3((unsigned)(STAGED_THREADS - (tab.any_bias ? 0 : 32 * BIAS_WARPS)), 1, 1);
     cfg.stream = p.stream;
     cudaLaunchAttribute attr[2];
