@@ -241,7 +241,8 @@ def run_ours(args):
 
     n = args.flat_params
     NA, NB = wl.CONFIG2.n_micro, wl.CONFIG3.n_micro
-    T, d_in, d_out = args.linear_tokens, wl.CONFIG3.d_in, wl.CONFIG3.d_out
+    T = args.linear_tokens
+    d_in, d_out = args.linear_dims if args.linear_dims else (wl.CONFIG3.d_in, wl.CONFIG3.d_out)
     seed_shift = 100000 * rank  # each rank owns its own replica's data (weak scaling)
 
     # phase A state and inputs
@@ -445,11 +446,11 @@ def run_ours(args):
 
 def load_traffic(n_flat, tokens, d_in, d_out):
     """Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the committed
-    ncu summaries, scaled to THIS run's launch.  The streaming kernels were captured on a
-    smaller buffer (their traffic is proportional to the element count); the figure is a lower
-    bound, because the last stores of the small captured launch were still in the L2 when it
-    ended.  The fused call's entry counts only for the shape it was captured on.  An entry is
-    dropped once one of the kernel's source files differs from those the counters were taken on."""
+    ncu summary (profiles/traffic.json: medians over the launches of a single-pass launch list of
+    the bench's own full-size step).  A run on another buffer size scales the streaming kernels'
+    figure by the element count (their traffic is proportional to it).  The fused call's entry
+    counts only for the shape it was captured on.  An entry is dropped once one of the kernel's
+    source files differs from those the counters were taken on."""
     import hashlib
     p = ROOT / "profiles" / "traffic.json"
     out = {}
@@ -472,10 +473,11 @@ def load_traffic(n_flat, tokens, d_in, d_out):
             continue
         if "captured_params" in ent:
             scale = n_flat / ent["captured_params"]
-            out[key] = {"bytes_per_launch": int(ent["captured_bytes"] * scale),
-                        "note": f"scaled from a {ent['captured_params']}-param capture "
-                                f"({ent['captured_bytes'] / ent['captured_params']:.2f} B/param); lower "
-                                "bound (stores still in the L2 when the captured launch ended)"}
+            per_param = ent["captured_bytes"] / ent["captured_params"]
+            note = (f"captured on launches of this size ({per_param:.2f} B/param)" if scale == 1.0 else
+                    f"scaled by the element count from a {ent['captured_params']}-param capture "
+                    f"({per_param:.2f} B/param)")
+            out[key] = {"bytes_per_launch": int(ent["captured_bytes"] * scale), "note": note}
         elif ent.get("shape") == [tokens, d_in, d_out]:
             out[key] = {"bytes_per_launch": int(ent["captured_bytes"]),
                         "note": "captured on this shape"}
@@ -1158,6 +1160,8 @@ def main():
     ap.add_argument("--linear-tokens", type=int, default=wl.CONFIG3.tokens,
                     help="tokens per micro-batch of the linear layer (default: the workload's 4096; "
                          "smaller values are for profiling the short-call kernel instance)")
+    ap.add_argument("--linear-dims", type=int, nargs=2, default=None, metavar=("D_IN", "D_OUT"),
+                    help="headline phase B on another layer shape (profiling runs; default 4096 4096)")
     ap.add_argument("--workload", default="headline", choices=["headline", "gpt2xl", "llama7b", "sweep", "small_tensors", "extensions", "oracle_timing", "wgrad_shapes", "launch_check"])
     ap.add_argument("--exchange", default="none", choices=["none", "allreduce", "sharded"],
                     help="N > 1: what the ranks exchange at the end of each mini-batch, inside the "

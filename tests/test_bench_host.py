@@ -32,7 +32,9 @@ def test_traffic_entry_is_scaled_to_the_run_and_dropped_when_a_source_changes(tm
     monkeypatch.setattr(bench, "ROOT", tmp_path)
     got = bench.load_traffic(5000, 64, 128, 256)
     assert got["fold_bf16"]["bytes_per_launch"] == 85000      # scaled by this run's size
-    assert "lower bound" in got["fold_bf16"]["note"] and "1000-param" in got["fold_bf16"]["note"]
+    assert "scaled" in got["fold_bf16"]["note"] and "1000-param" in got["fold_bf16"]["note"]
+    same = bench.load_traffic(1000, 64, 128, 256)             # the captured size itself: no scaling
+    assert same["fold_bf16"]["bytes_per_launch"] == 17000 and "of this size" in same["fold_bf16"]["note"]
     assert got["wgrad_fold"]["bytes_per_launch"] == 555
     assert "wgrad_fold" not in bench.load_traffic(5000, 64, 128, 512)   # another shape: no figure
     src.write_text("kernel v2")
