@@ -455,11 +455,11 @@ ADAMA_API adama_status adama_debug_wgrad_expire_wait(adama_ctx *ctx, const void 
  * 0 = automatic (the default).  epilogue: 1 = direct, 2 = staged through shared memory;
  * epi_warps: 4 or 8 (direct epilogue); box_loads: 1 = one TMA operation per 64-feature box
  * even where grouped loads apply; no_pdl: 1 = plain stream order instead of programmatic
- * dependent launch; tile_cols: width of the column tiles (a multiple of 32 up to 256).
+ * dependent launch.
  * Results do not depend on the choice beyond fp32 summation order inside the tensor cores
  * (none: the order over tokens is the same).  Errors: INVALID_ARG for any other value. */
 ADAMA_API adama_status adama_debug_set_wgrad_variant(adama_ctx *ctx, int epilogue, int epi_warps,
-                                                     int box_loads, int no_pdl, int tile_cols);
+                                                     int box_loads, int no_pdl);
 
 /* Diagnostics of the library's one-time set-up: bit 0 = the driver's tensor-map encoder has been
  * resolved (once per process), bit 1 = the fused kernel's attributes have been set on `device`

@@ -126,7 +126,7 @@ def load_library() -> ctypes.CDLL:
     L.adama_debug_set_status.argtypes = [vp, ctypes.c_uint, ctypes.c_uint, ctypes.c_uint, vp]
     L.adama_debug_wgrad_expire_wait.argtypes = [vp, vp, vp, ci, ci, ci, i64, i64, vp, vp, i64,
                                                 ctypes.c_uint64, vp]
-    L.adama_debug_set_wgrad_variant.argtypes = [vp, ci, ci, ci, ci, ci]
+    L.adama_debug_set_wgrad_variant.argtypes = [vp, ci, ci, ci, ci]
     L.adama_debug_setup_state.argtypes = [ci]
     L.adama_debug_setup_state.restype = ci
     L.adama_last_error.argtypes = [vp]
@@ -547,10 +547,10 @@ class AdamA:
             _stream_ptr(self.device)))
 
     def debug_set_wgrad_variant(self, epilogue: int = 0, epi_warps: int = 0, box_loads: int = 0,
-                                no_pdl: int = 0, tile_cols: int = 0) -> None:
+                                no_pdl: int = 0) -> None:
         """adama_debug_set_wgrad_variant (test hook: pins the fused kernel's instance)."""
         self._check(self._L.adama_debug_set_wgrad_variant(self._h, epilogue, epi_warps, box_loads,
-                                                          no_pdl, tile_cols))
+                                                          no_pdl))
 
     @property
     def launch_count(self) -> int:

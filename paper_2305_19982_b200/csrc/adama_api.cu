@@ -772,17 +772,15 @@ adama_status adama_debug_wgrad_expire_wait(adama_ctx *ctx, const void *X, const 
 }
 
 adama_status adama_debug_set_wgrad_variant(adama_ctx *ctx, int epilogue, int epi_warps,
-                                           int box_loads, int no_pdl, int tile_cols) {
+                                           int box_loads, int no_pdl) {
     if (!ctx) return ADAMA_ERR_INVALID_ARG;
     if (epilogue < 0 || epilogue > 2 || (epi_warps != 0 && epi_warps != 4 && epi_warps != 8) ||
-        (box_loads != 0 && box_loads != 1) || (no_pdl != 0 && no_pdl != 1) || tile_cols < 0 ||
-        tile_cols > 256 || tile_cols % 32)
+        (box_loads != 0 && box_loads != 1) || (no_pdl != 0 && no_pdl != 1))
         return fail(ctx, ADAMA_ERR_INVALID_ARG, "debug_set_wgrad_variant: value out of range");
     ctx->variant.epilogue = epilogue;
     ctx->variant.epi_warps = epi_warps;
     ctx->variant.box_loads = box_loads;
     ctx->variant.no_pdl = no_pdl;
-    ctx->variant.tile_cols = tile_cols;
     return ADAMA_OK;
 }
 

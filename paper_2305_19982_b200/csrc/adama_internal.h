@@ -98,7 +98,6 @@ struct WgradVariant {
     int epi_warps = 0;  // 4 or 8 epilogue warps (direct epilogue)
     int box_loads = 0;  // 1 = one TMA operation per 64-feature box even where grouped loads apply
     int no_pdl = 0;     // 1 = plain stream order instead of programmatic dependent launch
-    int tile_cols = 0;  // width of the column tiles (multiple of 32, <= 256)
 };
 constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;  // 2 s per device-side wait
 struct WgradArgs {

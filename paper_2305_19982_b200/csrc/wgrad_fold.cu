@@ -27,12 +27,19 @@
 //   warps 2..   epilogue: one or two warps per TMEM lane quarter (4 or 8 warps, chosen per
 //               launch; with two, each takes half of the tile's columns), in both CTAs
 // The 512 TMEM columns hold two 128x256 fp32 accumulators per CTA, so the epilogue of
-// tile i overlaps the main loop of tile i+1.  (A one-CTA variant, 128x256 tiles and a
-// 4-stage ring, is kept as a template instance for comparison.)
+// tile i overlaps the main loop of tile i+1.
 //   optional    two more warps that sum dY's columns into the bias moments (see the bias branch)
 // Calls of up to 2048 tokens run a second instance with a "staged" epilogue (see STAGED_RING):
 // 4 drain warps copy the accumulator to shared memory part by part, 8 streaming warps fold
 // the parts into m and v; the ring has 5 stages there.
+//
+// What bounds the main loop is the round trip of a ring stage, not the tensor core: a 2-CTA
+// tcgen05.mma of M = 256, N = 256, K = 16 takes 128 clocks (64 at N = 128), but a stage is held
+// from its TMA issue until tcgen05.commit reports its MMAs retired -- load latency + 512
+// clocks of MMAs + about 1600 clocks of commit latency + two wake-ups, some 3500 clocks against
+// the 6 x 512 that six stages cover.  Hence: every stage counts, a 128-column tile runs its
+// main loop no faster than a 256-column one (only 256 x 256 tiles are efficient), and the
+// barrier probes carry a suspend-time hint so that waiters wake without delay.
 //
 // Operand layout.  The contraction runs over tokens, the strided dimension of both
 // row-major inputs, so both operands are "MN-major": a TMA box of 64 features x 64

@@ -170,8 +170,7 @@ def test_every_kernel_instance_on_every_kind_of_shape(variant, T, d_in, d_out, p
 
 def test_variant_entry_rejects_values_out_of_range():
     opt = adama.AdamA()
-    for bad in (dict(epilogue=3), dict(epi_warps=6), dict(box_loads=2), dict(no_pdl=-1),
-                dict(tile_cols=48), dict(tile_cols=288)):
+    for bad in (dict(epilogue=3), dict(epi_warps=6), dict(box_loads=2), dict(no_pdl=-1)):
         with pytest.raises(adama.AdamAError) as e:
             opt.debug_set_wgrad_variant(**bad)
         assert e.value.status == adama.Status.ERR_INVALID_ARG
