@@ -589,7 +589,7 @@ def materialised_minibatch(stack, opt, n_micro, lr, inputs):
 
 
 def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, dev_index=0,
-                  layers_per_launch=1):
+                  layers_per_launch=1, blocks=None, n_micro_override=None):
     """GPT-2-XL- / Llama-7B-shaped stack, one mini-batch per step in the workload's own
     configuration (N = 8 / 16 micro-batches of 4096 tokens, layers back to front, fused
     weight-gradient fold per layer, one apply): time, TFLOP/s of the whole mini-batch, clocks,
@@ -602,11 +602,12 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
     dev = torch.device("cuda", dev_index)
     pk = peaks()
     if kind == "gpt2xl":
-        stack, tokens, n_micro, cfg_id = (gpt2xl_stack(wl.CONFIG4_BLOCKS, device=dev, biases=biases),
+        stack, tokens, n_micro, cfg_id = (gpt2xl_stack(blocks or wl.CONFIG4_BLOCKS, device=dev, biases=biases),
                                           wl.CONFIG4_TOKENS, wl.CONFIG4_N_MICRO, 4)
     else:
-        stack, tokens, n_micro, cfg_id = (llama7b_stack(wl.CONFIG5_BLOCKS, device=dev),
+        stack, tokens, n_micro, cfg_id = (llama7b_stack(blocks or wl.CONFIG5_BLOCKS, device=dev),
                                           wl.CONFIG5_TOKENS, wl.CONFIG5_N_MICRO, 5)
+    n_micro = n_micro_override or n_micro
     stack.w.normal_(0, 0.02, generator=torch.Generator(device=dev).manual_seed(wl.seed_for(cfg_id, 99)))
     # two seeded variants of X and dY per distinct width, reused across layers while timing
     widths = sorted({L.d_in for L in stack.layers} | {L.d_out for L in stack.layers})
@@ -699,7 +700,8 @@ def run_stack(args):
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(0)
     r = measure_stack(args.workload, args.steps, min(args.warmup, 2), biases=args.biases,
-                      layers_per_launch=args.layers_per_launch)
+                      layers_per_launch=args.layers_per_launch, blocks=args.stack_blocks,
+                      n_micro_override=args.stack_micro, with_gemm_pipeline=not args.stack_blocks)
     pk = peaks()
     line = {
         "metric": "adama_wgrad_fold_stack_TFLOPps", "value": r["TFLOPps"], "unit": "TFLOP/s", "n_gpus": 1,
@@ -1171,6 +1173,12 @@ def main():
     ap.add_argument("--layers-per-launch", type=int, default=1,
                     help="gpt2xl / llama7b workloads: consecutive layers folded by one grouped launch "
                          "(1 = one call per layer; 4 / 7 = one call per transformer block)")
+    ap.add_argument("--stack-blocks", type=int, default=None,
+                    help="gpt2xl / llama7b workloads: a shorter stack of that many blocks (profiling runs; "
+                         "default: the workload's 48 / 32)")
+    ap.add_argument("--stack-micro", type=int, default=None,
+                    help="gpt2xl / llama7b workloads: micro-batches per mini-batch (profiling runs; "
+                         "default: the workload's 8 / 16)")
     ap.add_argument("--no-stacks", action="store_true",
                     help="skip the two layer-stack workloads of the default line (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
