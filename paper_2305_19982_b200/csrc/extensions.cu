@@ -17,18 +17,9 @@ namespace {
 // Unroll factors from a sweep at 335 M elements on B200 (GB/s): sgdm fold 8/12/16/24 -> 5359/5731/
 // 5565/5753; sgdm apply 8/10/12/16 -> 6169/6077/6043/6015; coefficient 3/4/6/8 -> 4322/4669/5105/5366.
 constexpr int kThreads = 256;
-#ifndef ADAMA_SGDM_FOLD_UNROLL
-#define ADAMA_SGDM_FOLD_UNROLL 12
-#endif
-#ifndef ADAMA_SGDM_APPLY_UNROLL
-#define ADAMA_SGDM_APPLY_UNROLL 8
-#endif
-#ifndef ADAMA_COEF_UNROLL
-#define ADAMA_COEF_UNROLL 8
-#endif
-constexpr int kSgdmFoldUnroll = ADAMA_SGDM_FOLD_UNROLL;    // {g, buf} 128-bit groups in flight per thread
-constexpr int kSgdmApplyUnroll = ADAMA_SGDM_APPLY_UNROLL;  // {w, buf}
-constexpr int kCoefUnroll = ADAMA_COEF_UNROLL;             // {m, m_begin, v, v_adam}
+constexpr int kSgdmFoldUnroll = 12;   // {g, buf} 128-bit groups in flight per thread
+constexpr int kSgdmApplyUnroll = 8;   // {w, buf}
+constexpr int kCoefUnroll = 8;        // {m, m_begin, v, v_adam}
 
 template <typename G, int UNROLL>
 __global__ void __launch_bounds__(kThreads, 1)

@@ -11,28 +11,15 @@
 namespace adama {
 namespace {
 
-// Launch shape (overridable at build time for tuning sweeps).  Measured on B200 at 335 M
+// Launch shape.  Measured on B200 at 335 M
 // parameters: one fat CTA per SM with many independent 128-bit loads per thread beats
 // several thin ones -- fold 6.28 TB/s at (256 threads, unroll 6, 1 CTA/SM) against 6.03 at
 // (unroll 4, 4 CTAs/SM); apply 6.30 TB/s at (8 groups, 1 CTA/SM) against 5.81 at (4, 3).
-#ifndef ADAMA_FOLD_UNROLL
-#define ADAMA_FOLD_UNROLL 6
-#endif
-#ifndef ADAMA_FOLD_CTAS_PER_SM
-#define ADAMA_FOLD_CTAS_PER_SM 1
-#endif
-#ifndef ADAMA_APPLY_UNROLL
-#define ADAMA_APPLY_UNROLL 4
-#endif
-#ifndef ADAMA_APPLY_CTAS_PER_SM
-#define ADAMA_APPLY_CTAS_PER_SM 1
-#endif
-#ifndef ADAMA_STREAM_THREADS
-#define ADAMA_STREAM_THREADS 256
-#endif
-constexpr int kThreads = ADAMA_STREAM_THREADS;
-constexpr int kCtasPerSm = ADAMA_FOLD_CTAS_PER_SM;        // fold: 6 x (g, m, v) vectors in flight per thread
-constexpr int kApplyCtasPerSm = ADAMA_APPLY_CTAS_PER_SM;  // apply: 2 x 4 x (w, m, v) vectors = 96 data registers
+constexpr int kThreads = 256;
+constexpr int kFoldUnroll = 6;      // fold: 6 x (g, m, v) vectors in flight per thread
+constexpr int kApplyUnroll = 4;     // apply: 2 x 4 x (w, m, v) vectors = 96 data registers
+constexpr int kCtasPerSm = 1;
+constexpr int kApplyCtasPerSm = 1;
 
 template <typename G, int UNROLL>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
@@ -196,7 +183,7 @@ apply_scalar_kernel(float *__restrict__ w, float *__restrict__ m, float *__restr
 cudaError_t launch_fold(const void *grad, adama_dtype gdt, float *m, float *v, size_t n,
                         FoldConstants c, int sm_count, cudaStream_t stream) {
     if (n == 0) return cudaSuccess;
-    constexpr int U = ADAMA_FOLD_UNROLL;
+    constexpr int U = kFoldUnroll;
     const size_t n4 = n / 4;
     const bool vec = aligned(m, 16) && aligned(v, 16) && aligned(grad, gdt == ADAMA_F32 ? 16 : 8);
     if (gdt == ADAMA_F32) {
@@ -226,7 +213,7 @@ cudaError_t launch_apply(float *w, float *m, float *v, size_t n, ApplyConstants 
                          cudaStream_t stream, void *w_bf16_out) {
     __nv_bfloat16 *wb = static_cast<__nv_bfloat16 *>(w_bf16_out);
     if (n == 0) return cudaSuccess;
-    constexpr int U = ADAMA_APPLY_UNROLL;
+    constexpr int U = kApplyUnroll;
     const size_t n4 = n / 4;
     if (aligned(w, 16) && aligned(m, 16) && aligned(v, 16) && (!wb || aligned(wb, 8))) {
         unsigned grid = grid_for(n4, (size_t)kThreads * U, sm_count, kApplyCtasPerSm);

@@ -65,14 +65,9 @@
 namespace adama {
 namespace {
 
-#ifndef ADAMA_WGRAD_STAGES
-#define ADAMA_WGRAD_STAGES 6  // shared-memory ring depth of the CTA-pair kernel (build-time tunable)
-#endif
+constexpr int RING_STAGES = 6;  // shared-memory ring depth of the direct-epilogue instance
 constexpr int BN = 256;     // tile columns (d_out direction) = UMMA N
-#ifndef ADAMA_WGRAD_BK
-#define ADAMA_WGRAD_BK 64
-#endif
-constexpr int BK = ADAMA_WGRAD_BK;  // tokens per pipeline stage
+constexpr int BK = 64;      // tokens per pipeline stage
 constexpr int UMMA_K = 16;  // tokens per tcgen05.mma (bf16)
 constexpr int GROUP = 64;   // features per 128-byte swizzled row
 constexpr int BOX_BYTES = GROUP * BK * 2;               // 8192
@@ -91,10 +86,7 @@ constexpr int TMEM_COLS = 512;
 constexpr int ACC_STAGES = 2;
 constexpr int MAX_STAGES = 12;
 constexpr int SMEM_BAR_BYTES = 512;
-#ifndef ADAMA_WGRAD_BIAS_UNROLL
-#define ADAMA_WGRAD_BIAS_UNROLL 8
-#endif
-constexpr int BIAS_UNROLL = ADAMA_WGRAD_BIAS_UNROLL;  // 16-byte loads in flight per thread of a bias warp
+constexpr int BIAS_UNROLL = 8;  // 16-byte loads in flight per thread of a bias warp
 constexpr int BIAS_WARPS = 2;
 constexpr int SMEM_BIAS_BYTES = BIAS_WARPS * 32 * 4;
 
@@ -102,10 +94,7 @@ constexpr int SMEM_BIAS_BYTES = BIAS_WARPS * 32 * 4;
 // tile is first copied into shared memory, part by part (128 rows x PART_COLS fp32, two part
 // buffers, the rest of the shared memory stays with the ring), and separate streaming warps
 // fold the parts into m and v.
-#ifndef ADAMA_WGRAD_PART_COLS
-#define ADAMA_WGRAD_PART_COLS 64
-#endif
-constexpr int PART_COLS = ADAMA_WGRAD_PART_COLS;        // columns of one part of the tile copy
+constexpr int PART_COLS = 64;                           // columns of one part of the tile copy
 constexpr int PART_BYTES = 128 * PART_COLS * 4;         // 128 rows: 32 KB (64 columns) or 64 KB (128)
 constexpr int STAGED_RING = (224 * 1024 - 2 * PART_BYTES) / (32 * 1024);  // 5 or 3 stages
 constexpr int STAGED_DRAIN_WARPS = 4;   // tensor memory -> shared memory, one per lane quarter
@@ -127,7 +116,7 @@ struct Geo {
     static constexpr int B_STAGE_BYTES = B_BOXES * BOX_BYTES;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KB or 32 KB
     static constexpr int STAGES =
-        STAGED ? STAGED_RING : ADAMA_WGRAD_STAGES;
+        STAGED ? STAGED_RING : RING_STAGES;
     static constexpr int SMEM_EPI_OFF = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BAR_OFF = SMEM_EPI_OFF + (STAGED ? G_TILE_BYTES : EPI_BYTES);
     static constexpr int SMEM_BIAS_OFF = SMEM_BAR_OFF + SMEM_BAR_BYTES;
