@@ -405,14 +405,24 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_stacks:
         # the two layer-stack workloads in their stated configuration, 2 mini-batches each
         # ("_per_block": the linears of a transformer block folded by one grouped launch)
+        # ("_settled": context flag ADAMA_INPUTS_SETTLED -- a call's operand loads do not wait for the
+        # kernel before it; the stacks' inputs are complete long before, as the flag requires)
         stacks = {"gpt2xl": measure_stack("gpt2xl", 2, 1, dev_index=local),
                   "gpt2xl_per_block": measure_stack("gpt2xl", 2, 1, dev_index=local,
-                                                    with_gemm_pipeline=False, layers_per_launch=4)}
+                                                    with_gemm_pipeline=False, layers_per_launch=4),
+                  "gpt2xl_settled": measure_stack("gpt2xl", 2, 1, dev_index=local, with_gemm_pipeline=False,
+                                                  inputs_settled=True, with_memory=False),
+                  "gpt2xl_per_block_settled": measure_stack("gpt2xl", 2, 1, dev_index=local,
+                                                            with_gemm_pipeline=False, layers_per_launch=4,
+                                                            inputs_settled=True, with_memory=False)}
         free, _ = torch.cuda.mem_get_info()
         if free >= 100 * (1 << 30):
             stacks["llama7b"] = measure_stack("llama7b", 2, 1, dev_index=local)
             stacks["llama7b_per_block"] = measure_stack("llama7b", 2, 1, dev_index=local,
                                                         with_gemm_pipeline=False, layers_per_launch=7)
+            stacks["llama7b_settled"] = measure_stack("llama7b", 2, 1, dev_index=local,
+                                                      with_gemm_pipeline=False, inputs_settled=True,
+                                                      with_memory=False)
         else:
             stacks["llama7b"] = {"skipped": f"needs ~90 GB of free device memory, {free >> 30} GiB free"}
     if rank == 0:
@@ -589,13 +599,16 @@ def materialised_minibatch(stack, opt, n_micro, lr, inputs):
 
 
 def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, dev_index=0,
-                  layers_per_launch=1, blocks=None, n_micro_override=None):
+                  layers_per_launch=1, blocks=None, n_micro_override=None, inputs_settled=False,
+                  with_memory=True):
     """GPT-2-XL- / Llama-7B-shaped stack, one mini-batch per step in the workload's own
     configuration (N = 8 / 16 micro-batches of 4096 tokens, layers back to front, fused
     weight-gradient fold per layer, one apply): time, TFLOP/s of the whole mini-batch, clocks,
     peak device memory without a gradient buffer, with a per-layer one and with a whole-model one.
     layers_per_launch > 1: that many consecutive layers (a transformer block's linears) are folded
-    by one grouped launch, their X, dY released together after it."""
+    by one grouped launch, their X, dY released together after it.
+    inputs_settled: the context is created with ADAMA_INPUTS_SETTLED (the pooled X, dY are complete
+    long before any call, which is what the flag promises)."""
     import paper_2305_19982_b200 as adama
     from paper_2305_19982_b200.stack import gpt2xl_stack, llama7b_stack
 
@@ -615,7 +628,7 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
                   for k in range(2)] for d in widths}
     pool_y = {d: [wl.normal((tokens, d), 1e-2, torch.bfloat16, wl.seed_for(cfg_id, 0, k) + 50 + d, device=dev)
                   for k in range(2)] for d in widths}
-    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=dev_index)
+    opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=dev_index, inputs_settled=inputs_settled)
 
     def pooled(i, j, spec):
         return pool_x[spec.d_in][(i + j) & 1], pool_y[spec.d_out][(i + j) & 1]
@@ -660,7 +673,7 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
     del pool_x, pool_y
     torch.cuda.empty_cache()
     mem = {}
-    for mode in ("none", "layer"):
+    for mode in (("none", "layer") if with_memory else ()):
         torch.cuda.synchronize()
         torch.cuda.reset_peak_memory_stats(dev)
         if mode == "none":
@@ -675,18 +688,20 @@ def measure_stack(kind, steps, warmup, biases=False, with_gemm_pipeline=True, de
     out = {
         "workload": kind, "biases": bool(stack.biases), "layers": len(stack.layers),
         "params": stack.n_params, "tokens_per_micro_batch": tokens, "n_micro": n_micro,
-        "layers_per_launch": layers_per_launch, "steps": steps, "ms_per_minibatch": ms, "TFLOPps": tf,
+        "layers_per_launch": layers_per_launch, "inputs_settled_flag": bool(inputs_settled),
+        "steps": steps, "ms_per_minibatch": ms, "TFLOPps": tf,
         "frac_of_sustained_bf16": tf / pk["bf16_tflops_sustained"],
         "frac_of_burst_bf16": tf / pk["bf16_tflops"], "peak_source": pk["source"],
         "gpu_launches": int(launches), "clocks": clocks,
         "gemm_plus_fold_pipeline_ms_per_minibatch": ms_layer,
-        "peak_memory": {"state_bytes": state_bytes,
-                        "fused_no_gradient_buffer": mem["none"],
-                        "per_layer_gradient_released": mem["layer"],
-                        "whole_model_gradient_accumulation": mem["none"] + 4 * stack.n_params,
-                        "largest_layer_gradient_bytes": 4 * largest_layer,
-                        "note": "max_memory_allocated over one micro-batch with fresh X, dY per layer; "
-                                "the gradient-accumulation figure adds an fp32 gradient for every parameter"},
+        "peak_memory": None if not with_memory else {
+            "state_bytes": state_bytes,
+            "fused_no_gradient_buffer": mem["none"],
+            "per_layer_gradient_released": mem["layer"],
+            "whole_model_gradient_accumulation": mem["none"] + 4 * stack.n_params,
+            "largest_layer_gradient_bytes": 4 * largest_layer,
+            "note": "max_memory_allocated over one micro-batch with fresh X, dY per layer; "
+                    "the gradient-accumulation figure adds an fp32 gradient for every parameter"},
     }
     opt.close()
     del stack
@@ -701,7 +716,8 @@ def run_stack(args):
     torch.cuda.set_device(0)
     r = measure_stack(args.workload, args.steps, min(args.warmup, 2), biases=args.biases,
                       layers_per_launch=args.layers_per_launch, blocks=args.stack_blocks,
-                      n_micro_override=args.stack_micro, with_gemm_pipeline=not args.stack_blocks)
+                      n_micro_override=args.stack_micro, with_gemm_pipeline=not args.stack_blocks,
+                      inputs_settled=args.inputs_settled)
     pk = peaks()
     line = {
         "metric": "adama_wgrad_fold_stack_TFLOPps", "value": r["TFLOPps"], "unit": "TFLOP/s", "n_gpus": 1,
@@ -887,6 +903,10 @@ def run_wgrad_shapes(args):
             shapes.append((di, do))
     opt = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0)
     opt.begin_minibatch(4)
+    # a second context with ADAMA_INPUTS_SETTLED: a call's operand loads do not wait for the kernel
+    # before it (X, dY below are complete long before any call, as the flag requires)
+    opt_s = adama.AdamA(wl.BETA1, wl.BETA2, wl.EPS, device=0, inputs_settled=True)
+    opt_s.begin_minibatch(4)
 
     def timed(call, reps=20):
         for _ in range(3):
@@ -970,10 +990,15 @@ def run_wgrad_shapes(args):
         tf_cold = 2.0 * T * d_in * d_out / cold / 1e6
         us_model = timed_in_model(d_in, d_out, lambda mm, vv: opt.linear_wgrad_fold(X, dY, mm, vv))
         tf_model = 2.0 * T * d_in * d_out / us_model / 1e6
+        us_set = timed_in_model(d_in, d_out, lambda mm, vv: opt_s.linear_wgrad_fold(X, dY, mm, vv))
+        tf_set = 2.0 * T * d_in * d_out / us_set / 1e6
         rows.append({"d_in": d_in, "d_out": d_out, "tokens": T,
                      "in_model": {"us": us_model, "TFLOPps": tf_model,
                                   "frac_of_burst_peak": tf_model / pk["bf16_tflops"],
                                   "frac_of_sustained_peak": tf_model / pk["bf16_tflops_sustained"]},
+                     "in_model_inputs_settled": {"us": us_set, "TFLOPps": tf_set,
+                                                 "frac_of_burst_peak": tf_set / pk["bf16_tflops"],
+                                                 "frac_of_sustained_peak": tf_set / pk["bf16_tflops_sustained"]},
                      "back_to_back": {"us": us, "TFLOPps": tf,
                                       "frac_of_burst_peak": tf / pk["bf16_tflops"],
                                       "us_with_fused_bias": us_fused,
@@ -1018,13 +1043,16 @@ def run_wgrad_shapes(args):
         groups = [[(xs[di], ys[do], torch.zeros(di, do, device=dev), torch.zeros(di, do, device=dev))
                    for _, di, do in linears] for _ in range(copies)]
         res = {}
-        for mode in ("one_launch_per_block", "one_launch_per_layer"):
+        for mode in ("one_launch_per_block", "one_launch_per_layer",
+                     "one_launch_per_block_inputs_settled", "one_launch_per_layer_inputs_settled"):
+            o = opt_s if mode.endswith("_inputs_settled") else opt
+
             def run(g):
-                if mode == "one_launch_per_block":
-                    opt.linear_wgrad_fold_multi(g)
+                if mode.startswith("one_launch_per_block"):
+                    o.linear_wgrad_fold_multi(g)
                 else:
                     for item in g:
-                        opt.linear_wgrad_fold(*item)
+                        o.linear_wgrad_fold(*item)
             for g in groups:
                 run(g)
             torch.cuda.synchronize()
@@ -1045,6 +1073,8 @@ def run_wgrad_shapes(args):
         blocks.append({"block": name, "layers": [[di, do] for _, di, do in linears], "tokens": T, **res})
         del groups, xs, ys
     opt.sync_status()
+    opt_s.sync_status()
+    opt_s.close()
     print(json.dumps({"metric": "adama_wgrad_fold_per_shape", "token_sweep_4096x4096_l2_flushed": sweep,
                       "blocks_in_model": blocks, "unit": "us", "peak_tflops": pk["bf16_tflops"],
                       "peak_source": pk["source"],
@@ -1179,6 +1209,8 @@ def main():
     ap.add_argument("--stack-micro", type=int, default=None,
                     help="gpt2xl / llama7b workloads: micro-batches per mini-batch (profiling runs; "
                          "default: the workload's 8 / 16)")
+    ap.add_argument("--inputs-settled", action="store_true",
+                    help="gpt2xl / llama7b workloads: create the context with ADAMA_INPUTS_SETTLED")
     ap.add_argument("--no-stacks", action="store_true",
                     help="skip the two layer-stack workloads of the default line (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

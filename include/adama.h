@@ -76,6 +76,16 @@ typedef enum adama_dtype { ADAMA_F32 = 0, ADAMA_BF16 = 1 } adama_dtype;
  * `cuda_stream`, so that the copy (device to host) can run while later calls already stream the
  * next gradients in (host to device); see adama_apply_to_host for what the caller gives up. */
 #define ADAMA_ASYNC_COPYBACK 2u
+/* Promise about the inputs of the fused weight-gradient calls (adama_linear_wgrad_fold, _bias_fold,
+ * _multi): the X and dY handed to a call are NOT written by the kernel enqueued just before the
+ * call on the same stream -- they were complete earlier, as in a deferred weight-gradient pass or
+ * when the producing kernel is followed by some other kernel first.  The call's operand loads then
+ * do not wait for that previous kernel, so its first tiles run while the previous call's last,
+ * partly filled round of tiles still finishes (back-to-back calls on 1600 x 1600, 4096 tokens:
+ * 34.9 -> 22.5 us).  Everything else keeps its order: m, v (and the bias moments and dY reads of
+ * the bias warps) are touched only after the previous kernel has completed, so consecutive calls
+ * on the same layer stay correct.  Without the flag, the default, nothing is assumed. */
+#define ADAMA_INPUTS_SETTLED 4u
 
 typedef struct adama_config {
     double beta1;   /* in [0,1)                                    */

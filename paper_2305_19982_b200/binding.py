@@ -41,6 +41,7 @@ class Status(enum.IntEnum):
 F32, BF16 = 0, 1
 GRADS_PRESCALED = 1
 ASYNC_COPYBACK = 2
+INPUTS_SETTLED = 4
 
 
 class AdamAError(RuntimeError):
@@ -192,13 +193,14 @@ class AdamA:
     """
 
     def __init__(self, beta1=0.9, beta2=0.999, eps=1e-8, device=0, grads_prescaled=False,
-                 async_copyback=False):
+                 async_copyback=False, inputs_settled=False):
         self._L = load_library()
         self._h = ctypes.c_void_p()
         self.device = torch.device("cuda", int(device))
         cfg = _Config(beta1, beta2, eps, int(device),
                       (GRADS_PRESCALED if grads_prescaled else 0) |
-                      (ASYNC_COPYBACK if async_copyback else 0))
+                      (ASYNC_COPYBACK if async_copyback else 0) |
+                      (INPUTS_SETTLED if inputs_settled else 0))
         st = self._L.adama_init(ctypes.byref(self._h), ctypes.byref(cfg))
         if st != 0:
             self._h = ctypes.c_void_p()

@@ -101,7 +101,7 @@ cudaError_t join_copyback(adama_ctx *ctx, cudaStream_t stream) {
 bool config_ok(const adama_config *cfg) {
     return cfg && cfg->beta1 >= 0.0 && cfg->beta1 < 1.0 && cfg->beta2 >= 0.0 && cfg->beta2 < 1.0 &&
            cfg->eps >= 0.0 && isfinite(cfg->eps) && cfg->device >= 0 &&
-           (cfg->flags & ~(ADAMA_GRADS_PRESCALED | ADAMA_ASYNC_COPYBACK)) == 0;
+           (cfg->flags & ~(ADAMA_GRADS_PRESCALED | ADAMA_ASYNC_COPYBACK | ADAMA_INPUTS_SETTLED)) == 0;
 }
 
 adama_status check_fold_args(adama_ctx *ctx, const void *grad, adama_dtype gdt, float *m, float *v,
@@ -269,6 +269,7 @@ static adama_status wgrad_impl(adama_ctx *ctx, const void *X, const void *dY, in
     a.variant = ctx->variant;
     a.wait_limit_ns = wait_limit_ns;
     a.withhold_last_load = withhold_last_load;
+    a.inputs_settled = (ctx->cfg.flags & ADAMA_INPUTS_SETTLED) ? 1 : 0;
     const char *msg = "wgrad_fold";
     cudaError_t e = adama::launch_wgrad_fold(a, &msg);
     if (e != cudaSuccess) return cuda_fail(ctx, msg, e);
@@ -344,6 +345,7 @@ adama_status adama_linear_wgrad_fold_multi(adama_ctx *ctx, const adama_linear_it
         a.bias_m = it.m_bias;
         a.bias_v = it.v_bias;
         a.variant = ctx->variant;
+        a.inputs_settled = (ctx->cfg.flags & ADAMA_INPUTS_SETTLED) ? 1 : 0;
     }
     return ADAMA_OK;
 }

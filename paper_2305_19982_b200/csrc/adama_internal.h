@@ -118,6 +118,7 @@ struct WgradArgs {
     WgradVariant variant;
     unsigned long long wait_limit_ns = 0;  // 0 = kDefaultWaitLimitNs
     int withhold_last_load = 0;            // expiry test only: see adama_debug_wgrad_expire_wait
+    int inputs_settled = 0;                // ADAMA_INPUTS_SETTLED: X, dY not written by the kernel just before
 };
 // Returns cudaSuccess or the failing CUDA error; *msg (static string) says which step failed.
 cudaError_t launch_wgrad_fold(const WgradArgs &args, const char **msg);

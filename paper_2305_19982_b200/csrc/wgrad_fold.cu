@@ -442,7 +442,7 @@ __device__ __forceinline__ const WgradLayer *layer_of(const WgradTable &tab, int
 template <bool STAGED>
 __global__ void __launch_bounds__(STAGED ? STAGED_THREADS : MAX_THREADS, 1)
 wgrad_fold_kernel(const __grid_constant__ WgradTable tab, float a, float b, unsigned *status,
-                  unsigned long long wait_limit_ns, int withhold_last_load) {
+                  unsigned long long wait_limit_ns, int withhold_last_load, int inputs_settled) {
     using G = Geo<STAGED>;
     constexpr int STAGES = G::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -499,7 +499,10 @@ wgrad_fold_kernel(const __grid_constant__ WgradTable tab, float a, float b, unsi
     if (warp == 0) {
         // ---------------- TMA producer (one thread of every CTA) ----------------
         if (lane == 0) {
-            grid_dependency_wait();  // X and dY may come from the kernel just before this one
+            // X and dY may come from the kernel just before this one, unless the caller has
+            // promised otherwise (ADAMA_INPUTS_SETTLED): then the first tiles' loads and MMAs run
+            // beside that kernel's last round; m and v are still touched only after it
+            if (!inputs_settled) grid_dependency_wait();
             int stage = 0;
             uint32_t phase = 0;
             uint32_t armed = 0;        // bit s: stage s has been armed at least once
@@ -1269,7 +1272,7 @@ cudaError_t launch_wgrad_fold_multi(const WgradArgs *layers, int count, const ch
     cfg.numAttrs = p.variant.no_pdl ? 1 : 2;
     const unsigned long long limit = p.wait_limit_ns ? p.wait_limit_ns : kDefaultWaitLimitNs;
     return cudaLaunchKernelEx(&cfg, staged ? wgrad_fold_kernel<true> : wgrad_fold_kernel<false>, tab,
-                              p.c.a, p.c.b, p.status, limit, p.withhold_last_load);
+                              p.c.a, p.c.b, p.status, limit, p.withhold_last_load, p.inputs_settled);
 }
 
 cudaError_t launch_wgrad_fold(const WgradArgs &p, const char **msg) {

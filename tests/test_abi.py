@@ -96,3 +96,13 @@ def test_setup_bookkeeping_is_per_device_and_starts_empty():
         pytest.skip("another test in this process may already have launched on device 0")
     for dev in (0, 1, 7, 63, 64, 1000, -1):
         assert adama.debug_setup_state(dev) & 2 == 0
+
+
+def test_config_flags_known_and_unknown():
+    """The three configuration flags are accepted, any other bit is refused (host-only check)."""
+    for flags in (0, 1, 2, 4, 7):
+        adama.host_constants(0.9, 0.999, 1e-8, 4, 1, 1e-3, flags=flags)
+    for flags in (8, 16, 1 << 31):
+        with pytest.raises(adama.AdamAError) as e:
+            adama.host_constants(0.9, 0.999, 1e-8, 4, 1, 1e-3, flags=flags)
+        assert e.value.status == adama.Status.ERR_INVALID_ARG

@@ -408,3 +408,47 @@ def test_inputs_written_just_before_the_call_and_overwritten_just_after(T):
         opt.close()
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
     assert float(outs[0][1].max()) > 0
+
+
+def test_inputs_settled_flag_gives_the_same_results_back_to_back():
+    """ADAMA_INPUTS_SETTLED: the operand loads of a call do not wait for the kernel before it, so
+    the first tiles of a call run beside the last round of the previous one.  A run of calls back
+    to back -- the same layer four times in a row (its m, v carry from call to call, which the
+    epilogue's own wait must keep in order), layers with one tile and with more tiles than CTA
+    pairs, both epilogue forms, single and grouped launches -- must come out bit for bit as from
+    a context without the flag, and the repeated layer must match the oracle (integer inputs: exact).
+    All inputs are complete before the first call, which is what the flag promises."""
+    N = 4
+    specs = [(640, 1600, 1600), (192, 2560, 2048), (2304, 512, 768), (64, 136, 264), (2112, 640, 1280)]
+    data = []
+    for k, (T, d_in, d_out) in enumerate(specs):
+        Xs = [wl.small_integers((T, d_in), 3, torch.bfloat16, 900 + 10 * k + i) for i in range(N)]
+        Ys = [wl.small_integers((T, d_out), 3, torch.bfloat16, 950 + 10 * k + i) for i in range(N)]
+        data.append((Xs, Ys, [x.cuda() for x in Xs], [y.cuda() for y in Ys]))
+    torch.cuda.synchronize()
+    results = []
+    for settled in (False, True):
+        opt = adama.AdamA(inputs_settled=settled)
+        opt.begin_minibatch(N)
+        states = [(torch.zeros(d_in, d_out, device="cuda"), torch.zeros(d_in, d_out, device="cuda"))
+                  for (_, d_in, d_out) in specs]
+        for rep in range(2):
+            for i in range(N):                       # the same layer, call after call
+                opt.linear_wgrad_fold(data[0][2][i], data[0][3][i], *states[0])
+            for k in range(1, len(specs)):           # other layers, one launch each
+                opt.linear_wgrad_fold(data[k][2][rep], data[k][3][rep], *states[k])
+            opt.linear_wgrad_fold_multi([(data[k][2][2 + rep], data[k][3][2 + rep], *states[k])
+                                         for k in range(1, len(specs))])   # and grouped
+        opt.sync_status()
+        results.append(states)
+        opt.close()
+    for (m0, v0), (m1, v1) in zip(*results):
+        assert torch.equal(m0, m1) and torch.equal(v0, v1)
+    T, d_in, d_out = specs[0]
+    orc = AdamAOracle(np.zeros((d_in, d_out)))
+    orc.begin_minibatch(N)
+    for rep in range(2):
+        for i in range(N):
+            orc.fold_linear(f64(data[0][0][i]), f64(data[0][1][i]))
+    assert_close(f64(results[1][0][0]), orc.m, TOL_EXACT, "m, settled inputs", elementwise=True)
+    assert_close(f64(results[1][0][1]), orc.v, TOL_EXACT, "v, settled inputs", elementwise=True)
