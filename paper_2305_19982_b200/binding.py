@@ -190,6 +190,10 @@ class AdamA:
 
     Methods mirror the C ABI one to one; tensors are torch CUDA tensors owned by
     the caller, work is queued on torch's current stream of the context's device.
+    The keyword flags are adama_config.flags: grads_prescaled = ADAMA_GRADS_PRESCALED,
+    async_copyback = ADAMA_ASYNC_COPYBACK, inputs_settled = ADAMA_INPUTS_SETTLED (the caller
+    promises that X, dY of the fused calls are not written by the kernel enqueued just before
+    the call; see include/adama.h).
     """
 
     def __init__(self, beta1=0.9, beta2=0.999, eps=1e-8, device=0, grads_prescaled=False,
