@@ -168,7 +168,11 @@ ADAMA_API adama_status adama_linear_wgrad_fold(adama_ctx *ctx, const void *X, co
  * epilogue are paid once per launch instead of once per layer.  The price is that the layers'
  * X and dY must all be alive until the launch has run (they can be released one launch later
  * than with per-layer calls; m, v and the weight gradient are unaffected: there still is no
- * gradient buffer).  The layers must not share m or v storage.
+ * gradient buffer).  The layers must not share m or v storage, and no X or dY may overlap any
+ * layer's m, v or bias moments.  A call with more than 8 layers makes several launches; from its
+ * second launch on the operand loads do not wait for the call's own previous launch (which
+ * writes no X or dY), so consecutive launches overlap at their seams as with
+ * ADAMA_INPUTS_SETTLED.
  *   items : `count` descriptions in HOST memory, read before the call returns; per item the
  *           arguments of adama_linear_wgrad_fold, plus m_bias / v_bias (both null or both set).
  * Items with tokens == 0 are skipped.  Errors: as adama_linear_wgrad_fold, reported for the

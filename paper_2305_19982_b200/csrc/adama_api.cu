@@ -315,12 +315,17 @@ adama_status adama_linear_wgrad_fold_multi(adama_ctx *ctx, const adama_linear_it
     DeviceGuard guard(ctx->cfg.device);
     adama::WgradArgs batch[adama::kMaxWgradLayers];
     int k = 0;
+    bool first_launch = true;
     for (int i = 0; i <= count; ++i) {
         if ((i == count || k == adama::kMaxWgradLayers) && k > 0) {
+            // From the call's second launch on, the kernel just before is this call's own previous
+            // launch, which writes only m, v and bias moments: the operand loads need not wait for it.
+            if (!first_launch) batch[0].inputs_settled = 1;
             const char *msg = "wgrad_fold_multi";
             cudaError_t e = adama::launch_wgrad_fold_multi(batch, k, &msg);
             if (e != cudaSuccess) return cuda_fail(ctx, msg, e);
             ctx->launches += 1;
+            first_launch = false;
             k = 0;
         }
         if (i == count) break;
